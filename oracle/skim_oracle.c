@@ -1,0 +1,495 @@
+/*
+ * skim_oracle.c -- plain CPU oracle for the SKIM row-clustering path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, obviously-correct statement of
+ * what the path computes.  It shares no code with the CUDA implementation and must
+ * never be used by it: only the test-suite, the smoke check and the benchmark's
+ * CPU-baseline leg may build, load or call it.
+ *
+ * What it follows (SKIM, arXiv 2412.04180):
+ *   - weighted 1-D K-means of one weight row with per-element importance, objective
+ *     sum_j g_ij (w_ij - wq_ij)^2                       -- Section 3.2 (sensitivity,
+ *     diagonal form) and Section 4.1 (S-diag for K-means); Algorithm 3, error
+ *     pre-recording loop and final clustering loop.
+ *   - greedy bit allocation                               -- Section 4.2, Algorithm 1.
+ *   - scaling vector  Wq = Quant(W * alpha^-1) * alpha    -- Section 4.3, Algorithm 2.
+ *   - packing rows grouped by bit-width                   -- Section 4.2, last paragraph.
+ *
+ * Readings where the paper is silent (kept identical on the CUDA side):
+ *   - init: centroid j of k = sorted_row[ floor((2j+1) m / (2k)) ] (index quantiles).
+ *   - exactly `iters` (assign, update) pairs, then one more assign against the final
+ *     centroids; err and labels use that last assignment.
+ *   - assign: nearest centroid by a plain scan j = 0..k-1.  A tie between two different
+ *     centroid values (an element exactly at their midpoint) goes to the lower value; a tie
+ *     between equal-valued centroids goes to the copy on the element's side (the highest
+ *     copy for an element above that value, else the lowest).  With ascending centroids
+ *     this is the 1-D quantiser rule  label = #{ j : (c_j + c_{j+1})/2 < x }  and it keeps
+ *     the centroids ascending through every update.
+ *   - update: c_j = sum g x / sum g over the members; a cluster whose weight sum is
+ *     not > 0 keeps its centroid.
+ *   - if the row has D <= k distinct values: centroids are those values ascending, padded
+ *     with the largest; err = 0; no iterations.
+ *   - the error recorded in the table is the K-means objective itself (diagonal form).
+ *   - between iterations the centroids are held as IEEE binary32 (the precision of the
+ *     library's centroid output); all sums are binary64.  `round_fp32 = 0` keeps them
+ *     binary64 instead (used by the textbook pins).
+ *   - a scaled row is clustered on x~ = float(w) * r_j with r_j = 1.0f / s_j, the product
+ *     taken in binary32, so that both sides cluster bit-identical numbers.
+ *
+ * Parity pins: every function here is pinned by tests that do not call the CUDA path
+ * (closed forms, brute force, exact DP, library K-means, finite differences).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define SKIM_ORACLE_MAX_K 256
+
+/* ------------------------------------------------------------------ number formats */
+
+/* IEEE binary16 bit pattern -> float, exact. */
+static float half_bits_to_float(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) & 1u;
+    uint32_t exp = (uint32_t)(h >> 10) & 0x1fu;
+    uint32_t man = (uint32_t)h & 0x3ffu;
+    float v;
+    if (exp == 0) {
+        v = ldexpf((float)man, -24);                 /* subnormal or zero */
+    } else if (exp == 31) {
+        v = man ? NAN : INFINITY;
+    } else {
+        v = ldexpf((float)(man | 0x400u), (int)exp - 25);
+    }
+    return sign ? -v : v;
+}
+
+/* float -> IEEE binary16 bit pattern, round to nearest even. */
+static uint16_t float_to_half_bits(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    uint32_t sign = (u >> 16) & 0x8000u;
+    uint32_t mag = u & 0x7fffffffu;
+    if (mag >= 0x7f800000u) {                        /* inf or nan */
+        return (uint16_t)(sign | 0x7c00u | (mag > 0x7f800000u ? 0x200u : 0u));
+    }
+    double a = fabs((double)f);
+    if (a >= 65520.0) return (uint16_t)(sign | 0x7c00u);   /* rounds to inf */
+    if (a < ldexp(1.0, -14)) {
+        /* subnormal half: multiples of 2^-24 */
+        double q = nearbyint(a * ldexp(1.0, 24));   /* default mode: ties to even */
+        return (uint16_t)(sign | (uint32_t)q);      /* q == 1024 lands on the smallest normal */
+    }
+    int e;
+    double fr = frexp(a, &e);                        /* a = fr * 2^e, fr in [0.5, 1) */
+    double q = nearbyint(fr * 2048.0);               /* 11 significant bits */
+    if (q == 2048.0) { q = 1024.0; e += 1; }
+    uint32_t he = (uint32_t)(e - 1 + 15);
+    return (uint16_t)(sign | (he << 10) | ((uint32_t)q - 1024u));
+}
+
+uint16_t skim_oracle_float_to_half(float f) { return float_to_half_bits(f); }
+float skim_oracle_half_to_float(uint16_t h) { return half_bits_to_float(h); }
+
+/* The value that is clustered for element (., j): the fp16 weight, times r_j = 1.0f/s_j in
+ * binary32 when a scale vector is given (Section 4.3: W * alpha^-1). */
+static double clustered_value(uint16_t w, const float *s, int64_t j)
+{
+    float x = half_bits_to_float(w);
+    if (s) {
+        volatile float r = 1.0f / s[j];
+        volatile float p = x * r;
+        x = p;
+    }
+    if (x == 0.0f) x = 0.0f;                          /* -0 and +0 are one value */
+    return (double)x;
+}
+
+static int cmp_double(const void *a, const void *b)
+{
+    double x = *(const double *)a, y = *(const double *)b;
+    return (x > y) - (x < y);
+}
+
+/* ------------------------------------------------------------------ one row, one k */
+
+/* Nearest centroid, plain scan over ascending centroids.  Equal distances: keep the earlier
+ * centroid unless the later one lies below x (then the two are equal-valued copies below x,
+ * or x sits past both), see the tie rule in the header. */
+static int nearest_centroid(double x, const double *c, int k)
+{
+    int best = 0;
+    double bd = fabs(x - c[0]);
+    for (int j = 1; j < k; ++j) {
+        double d = fabs(x - c[j]);
+        if (d < bd || (d == bd && c[j] < x)) { bd = d; best = j; }
+    }
+    return best;
+}
+
+static double objective(const double *x, const double *g, int64_t m, const double *c, const int32_t *label)
+{
+    double e = 0.0;
+    for (int64_t j = 0; j < m; ++j) {
+        double d = x[j] - c[label[j]];
+        e += g[j] * d * d;
+    }
+    return e;
+}
+
+/*
+ * Weighted 1-D K-means of one row (Algorithm 3, the Kmeans(W_i, weights=G_i, 2^b) call,
+ * objective of Section 3.2's diagonal form).
+ *   x, g      [m]   values to cluster and their importance (g >= 0)
+ *   c         [k]   out: centroids, ascending
+ *   label     [m]   out: cluster index of every element (final assignment)
+ *   err             out: sum g (x - c[label])^2 for the final assignment
+ *   trace           out, optional [2*iters+1]: objective after every assign and every update
+ *   n_distinct      out, optional: number of distinct values, capped at k+1
+ * Returns 0, or -1 on bad arguments / allocation failure.
+ */
+int skim_oracle_kmeans_row(const double *x, const double *g, int64_t m, int k, int iters,
+                           int round_fp32, double *c, int32_t *label, double *err,
+                           double *trace, int *n_distinct)
+{
+    if (m <= 0 || k <= 0 || k > SKIM_ORACLE_MAX_K || iters < 0) return -1;
+    double *sorted = (double *)malloc((size_t)m * sizeof(double));
+    if (!sorted) return -1;
+    memcpy(sorted, x, (size_t)m * sizeof(double));
+    qsort(sorted, (size_t)m, sizeof(double), cmp_double);
+
+    /* distinct values (up to k+1 of them) */
+    double distinct[SKIM_ORACLE_MAX_K + 1];
+    int D = 0;
+    for (int64_t j = 0; j < m && D <= k; ++j) {
+        if (j == 0 || sorted[j] != sorted[j - 1]) distinct[D++] = sorted[j];
+    }
+    if (n_distinct) *n_distinct = D;
+
+    if (D <= k) {
+        /* every value gets its own centroid: zero error, no iterations */
+        for (int j = 0; j < k; ++j) c[j] = distinct[j < D ? j : D - 1];
+        for (int64_t j = 0; j < m; ++j) label[j] = nearest_centroid(x[j], c, k);
+        *err = 0.0;
+        if (trace) for (int t = 0; t < 2 * iters + 1; ++t) trace[t] = 0.0;
+        free(sorted);
+        return 0;
+    }
+
+    /* index-quantile init */
+    for (int j = 0; j < k; ++j) {
+        int64_t idx = ((int64_t)(2 * j + 1) * m) / (int64_t)(2 * k);
+        c[j] = sorted[idx];
+    }
+    free(sorted);
+
+    for (int it = 0; it < iters; ++it) {
+        double sg[SKIM_ORACLE_MAX_K], sgx[SKIM_ORACLE_MAX_K];
+        for (int j = 0; j < k; ++j) { sg[j] = 0.0; sgx[j] = 0.0; }
+        /* assign */
+        for (int64_t j = 0; j < m; ++j) {
+            int l = nearest_centroid(x[j], c, k);
+            label[j] = l;
+            sg[l] += g[j];
+            sgx[l] += g[j] * x[j];
+        }
+        if (trace) trace[2 * it] = objective(x, g, m, c, label);
+        /* update */
+        for (int j = 0; j < k; ++j) {
+            if (sg[j] > 0.0) {
+                double cj = sgx[j] / sg[j];
+                c[j] = round_fp32 ? (double)(float)cj : cj;
+            }
+        }
+        if (trace) trace[2 * it + 1] = objective(x, g, m, c, label);
+    }
+    /* final assignment against the final centroids */
+    for (int64_t j = 0; j < m; ++j) label[j] = nearest_centroid(x[j], c, k);
+    *err = objective(x, g, m, c, label);
+    if (trace) trace[2 * iters] = *err;
+    return 0;
+}
+
+/* ------------------------------------------------------------------ all rows, all bit-widths */
+
+static int check_bit_set(const int *bit_set, int n_bits)
+{
+    if (!bit_set || n_bits <= 0) return -1;
+    for (int b = 0; b < n_bits; ++b) {
+        if (bit_set[b] < 1 || bit_set[b] > 8) return -1;
+        if (b && bit_set[b] != bit_set[b - 1] + 1) return -1;
+    }
+    return 0;
+}
+
+/*
+ * Error pre-recording (Algorithm 3, the double loop over rows and candidate bit-widths) and,
+ * with `row_bits`, the final clustering at the allocated width (Algorithm 3, second row loop).
+ *   W          fp16 bit patterns, row-major, leading dimension ld
+ *   importance float, same layout
+ *   s          optional scale vector [cols] (NULL = none)
+ *   row_bits   optional [rows]: cluster row i only at bit-width row_bits[i]; other slots untouched
+ *   centroids  out [rows][sum_b 2^b] double, bit-width blocks in bit_set order
+ *   codes      out, optional [n_bits][rows][cols] uint8 labels
+ *   err        out [rows][n_bits] double
+ *   trace      out, optional [rows][n_bits][2*iters+1]
+ */
+int skim_oracle_cluster_rows(const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                             int64_t ld, const float *s, const uint8_t *row_bits,
+                             const int *bit_set, int n_bits, int iters, int round_fp32,
+                             double *centroids, uint8_t *codes, double *err, double *trace)
+{
+    if (!W || !importance || rows < 0 || cols <= 0 || ld < cols || iters < 0) return -1;
+    if (check_bit_set(bit_set, n_bits)) return -1;
+    int sumk = 0;
+    for (int b = 0; b < n_bits; ++b) sumk += 1 << bit_set[b];
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < rows; ++i) {
+        double *x = (double *)malloc((size_t)cols * sizeof(double));
+        double *g = (double *)malloc((size_t)cols * sizeof(double));
+        int32_t *label = (int32_t *)malloc((size_t)cols * sizeof(int32_t));
+        if (!x || !g || !label) {
+            failed = 1;
+        } else {
+            for (int64_t j = 0; j < cols; ++j) {
+                x[j] = clustered_value(W[i * ld + j], s, j);
+                g[j] = (double)importance[i * ld + j];
+            }
+            int off = 0;
+            for (int b = 0; b < n_bits; ++b) {
+                int k = 1 << bit_set[b];
+                if (!row_bits || row_bits[i] == bit_set[b]) {
+                    double e = 0.0;
+                    double *tr = trace ? trace + ((size_t)i * n_bits + b) * (size_t)(2 * iters + 1) : NULL;
+                    if (skim_oracle_kmeans_row(x, g, cols, k, iters, round_fp32,
+                                               centroids + (size_t)i * sumk + off, label, &e, tr, NULL))
+                        failed = 1;
+                    err[(size_t)i * n_bits + b] = e;
+                    if (codes) {
+                        uint8_t *dst = codes + ((size_t)b * rows + i) * (size_t)cols;
+                        for (int64_t j = 0; j < cols; ++j) dst[j] = (uint8_t)label[j];
+                    }
+                }
+                off += k;
+            }
+        }
+        free(x); free(g); free(label);
+    }
+    return failed ? -1 : 0;
+}
+
+/* ------------------------------------------------------------------ greedy bit allocation */
+
+/*
+ * Algorithm 1 (Section 4.2).  All rows start at b_min; the row whose next bit removes the
+ * most error (E[i,b_i] - E[i,b_i+1], lowest row index on ties) is raised by one bit, until
+ * the total reaches T = floor(rows * budget + 1e-6).  Gains are differences of the float
+ * table entries taken in binary64.
+ *   err   [rows][n_bits] float, column b is bit-width b_min + b
+ *   bits  out [rows]
+ *   total out: T
+ * Returns 0, -1 on bad arguments, -2 if the budget is outside [b_min, b_max].
+ */
+int skim_oracle_allocate_bits(const float *err, int64_t rows, int n_bits, int b_min, double budget,
+                              uint8_t *bits, int64_t *total)
+{
+    if (!err || !bits || rows <= 0 || n_bits <= 0 || b_min < 1) return -1;
+    int b_max = b_min + n_bits - 1;
+    int64_t T = (int64_t)floor((double)rows * budget + 1e-6);
+    int64_t K = T - rows * (int64_t)b_min;
+    if (K < 0 || K > rows * (int64_t)(b_max - b_min)) return -2;
+    for (int64_t i = 0; i < rows; ++i) bits[i] = (uint8_t)b_min;
+    for (int64_t step = 0; step < K; ++step) {
+        int64_t best = -1;
+        double best_gain = 0.0;
+        for (int64_t i = 0; i < rows; ++i) {
+            if (bits[i] >= b_max) continue;
+            int b = bits[i] - b_min;
+            double gain = (double)err[i * n_bits + b] - (double)err[i * n_bits + b + 1];
+            if (best < 0 || gain > best_gain) { best = i; best_gain = gain; }
+        }
+        bits[best] += 1;
+    }
+    if (total) *total = T;
+    return 0;
+}
+
+/* ------------------------------------------------------------------ emission */
+
+/* Words in one packed row of `cols` codes of `b` bits: ceil(cols*b/32), rounded up to 4 words. */
+int64_t skim_oracle_row_stride_words(int64_t cols, int b)
+{
+    int64_t w = (cols * (int64_t)b + 31) / 32;
+    return (w + 3) / 4 * 4;
+}
+
+/*
+ * Final codebook and code emission (Algorithm 3: labels and centroids at the allocated width;
+ * Section 4.2: rows of equal width are gathered and packed together).
+ *   bits        [rows] allocated width of every row
+ *   centroids   [rows][sum_b 2^b] float, as produced by the clustering (only the block of the
+ *               row's own width is read)
+ *   packed      out: for width b (ascending) the rows of that width in ascending row index,
+ *               each a little-endian bitstream (element j in bits [j*b, (j+1)*b)) stored as
+ *               32-bit words with stride skim_oracle_row_stride_words(cols, b); zero padded
+ *   row_order   out [rows]: source row of every packed row
+ *   group_start out [n_bits+1]: first packed-row index of every width group
+ *   group_word  out [n_bits+1]: word offset of every width group inside `packed`
+ *   lut         out [rows][2^b_max] fp16 bit patterns, entries beyond 2^b_i repeat the last
+ *   codes       out, optional [rows][cols] unpacked labels
+ */
+int skim_oracle_emit(const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *s,
+                     const uint8_t *bits, const float *centroids, const int *bit_set, int n_bits,
+                     uint32_t *packed, int32_t *row_order, int64_t *group_start, int64_t *group_word,
+                     uint16_t *lut, uint8_t *codes)
+{
+    if (!W || !bits || !centroids || rows <= 0 || cols <= 0 || ld < cols) return -1;
+    if (check_bit_set(bit_set, n_bits)) return -1;
+    int sumk = 0, kmax = 1 << bit_set[n_bits - 1];
+    for (int b = 0; b < n_bits; ++b) sumk += 1 << bit_set[b];
+
+    /* group rows by width, ascending width then ascending row */
+    int64_t pos = 0, word = 0;
+    for (int b = 0; b < n_bits; ++b) {
+        group_start[b] = pos;
+        group_word[b] = word;
+        int64_t cnt = 0;
+        for (int64_t i = 0; i < rows; ++i) {
+            if (bits[i] == bit_set[b]) { row_order[pos + cnt] = (int32_t)i; ++cnt; }
+        }
+        pos += cnt;
+        word += cnt * skim_oracle_row_stride_words(cols, bit_set[b]);
+    }
+    group_start[n_bits] = pos;
+    group_word[n_bits] = word;
+    if (pos != rows) return -3;                       /* some row has a width outside bit_set */
+    memset(packed, 0, (size_t)word * sizeof(uint32_t));
+
+    for (int b = 0; b < n_bits; ++b) {
+        int width = bit_set[b], k = 1 << width, off = 0;
+        for (int u = 0; u < b; ++u) off += 1 << bit_set[u];
+        int64_t stride = skim_oracle_row_stride_words(cols, width);
+        for (int64_t p = group_start[b]; p < group_start[b + 1]; ++p) {
+            int64_t i = row_order[p];
+            double c[SKIM_ORACLE_MAX_K];
+            for (int j = 0; j < k; ++j) c[j] = (double)centroids[(size_t)i * sumk + off + j];
+            uint32_t *dst = packed + group_word[b] + (p - group_start[b]) * stride;
+            for (int64_t j = 0; j < cols; ++j) {
+                double x = clustered_value(W[i * ld + j], s, j);
+                uint32_t code = (uint32_t)nearest_centroid(x, c, k);
+                if (codes) codes[(size_t)i * cols + j] = (uint8_t)code;
+                int64_t bit = j * width;
+                for (int t = 0; t < width; ++t) {
+                    if ((code >> t) & 1u) dst[(bit + t) / 32] |= 1u << ((bit + t) % 32);
+                }
+            }
+            for (int j = 0; j < kmax; ++j) {
+                float cv = centroids[(size_t)i * sumk + off + (j < k ? j : k - 1)];
+                lut[(size_t)i * kmax + j] = float_to_half_bits(cv);
+            }
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ scaling-vector update */
+
+/*
+ * Loss and gradient of the scaling vector with the labels held fixed (Algorithm 2, inner
+ * repeat: c = calc_centroids(W * alpha^-1, L); Wq = replace(c, L) * alpha; loss = Err(W, Wq)),
+ * with the diagonal error  loss = sum_ij g_ij (W_ij - alpha_j c_{i,l_ij})^2  and importance-
+ * weighted centroids  c_ik = sum_{j in k} g_ij W_ij / alpha_j  /  sum_{j in k} g_ij.
+ *   labels [rows][cols] uint8,  alpha [cols] double,  grad out [cols] (may be NULL)
+ */
+int skim_oracle_scale_loss_grad(const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                                int64_t ld, const uint8_t *labels, const double *alpha,
+                                double *loss_out, double *grad)
+{
+    if (!W || !importance || !labels || !alpha || rows <= 0 || cols <= 0 || ld < cols) return -1;
+    double loss = 0.0;
+    if (grad) for (int64_t j = 0; j < cols; ++j) grad[j] = 0.0;
+    for (int64_t i = 0; i < rows; ++i) {
+        double G[SKIM_ORACLE_MAX_K], S[SKIM_ORACLE_MAX_K], c[SKIM_ORACLE_MAX_K], R[SKIM_ORACLE_MAX_K];
+        for (int k = 0; k < SKIM_ORACLE_MAX_K; ++k) { G[k] = 0.0; S[k] = 0.0; c[k] = 0.0; R[k] = 0.0; }
+        for (int64_t j = 0; j < cols; ++j) {
+            double w = (double)half_bits_to_float(W[i * ld + j]);
+            double g = (double)importance[i * ld + j];
+            int l = labels[i * cols + j];
+            G[l] += g;
+            S[l] += g * w / alpha[j];
+        }
+        for (int k = 0; k < SKIM_ORACLE_MAX_K; ++k) if (G[k] > 0.0) c[k] = S[k] / G[k];
+        for (int64_t j = 0; j < cols; ++j) {
+            double w = (double)half_bits_to_float(W[i * ld + j]);
+            double g = (double)importance[i * ld + j];
+            int l = labels[i * cols + j];
+            double r = w - alpha[j] * c[l];
+            loss += g * r * r;
+            R[l] += g * r * alpha[j];
+        }
+        if (grad) {
+            for (int64_t j = 0; j < cols; ++j) {
+                double w = (double)half_bits_to_float(W[i * ld + j]);
+                double g = (double)importance[i * ld + j];
+                int l = labels[i * cols + j];
+                double r = w - alpha[j] * c[l];
+                double d = -2.0 * g * r * c[l];
+                if (G[l] > 0.0) d += 2.0 * R[l] * g * w / (alpha[j] * alpha[j] * G[l]);
+                grad[j] += d;
+            }
+        }
+    }
+    *loss_out = loss;
+    return 0;
+}
+
+/*
+ * `steps` Adam updates of alpha with the labels fixed (Section 5.1: Adam, learning rate lr0,
+ * multiplied by `decay` every `decay_every` steps; default betas 0.9 / 0.999, eps 1e-8).
+ *   alpha      in/out [cols]
+ *   loss_trace out, optional [steps]: loss at the alpha each step started from
+ */
+int skim_oracle_scale_update(const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                             int64_t ld, const uint8_t *labels, double *alpha, int steps, double lr0,
+                             double decay, int decay_every, double beta1, double beta2, double eps,
+                             double *loss_trace)
+{
+    if (steps < 0 || decay_every <= 0) return -1;
+    double *m1 = (double *)calloc((size_t)cols, sizeof(double));
+    double *m2 = (double *)calloc((size_t)cols, sizeof(double));
+    double *grad = (double *)malloc((size_t)cols * sizeof(double));
+    if (!m1 || !m2 || !grad) { free(m1); free(m2); free(grad); return -1; }
+    int rc = 0;
+    for (int t = 0; t < steps && !rc; ++t) {
+        double loss;
+        rc = skim_oracle_scale_loss_grad(W, importance, rows, cols, ld, labels, alpha, &loss, grad);
+        if (loss_trace) loss_trace[t] = loss;
+        double lr = lr0 * pow(decay, (double)(t / decay_every));
+        double bc1 = 1.0 - pow(beta1, (double)(t + 1));
+        double bc2 = 1.0 - pow(beta2, (double)(t + 1));
+        for (int64_t j = 0; j < cols; ++j) {
+            m1[j] = beta1 * m1[j] + (1.0 - beta1) * grad[j];
+            m2[j] = beta2 * m2[j] + (1.0 - beta2) * grad[j] * grad[j];
+            double mh = m1[j] / bc1, vh = m2[j] / bc2;
+            alpha[j] -= lr * mh / (sqrt(vh) + eps);
+        }
+    }
+    free(m1); free(m2); free(grad);
+    return rc;
+}
+
+int skim_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,188 @@
+"""ctypes binding of the CPU oracle (``skim_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the test-suite, the smoke check and the
+benchmark's CPU-baseline leg.  It imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "skim_oracle.c")
+_LIB = os.path.join(_HERE, "libskim_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over rows only); returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-std=c11", "-O2", "-fno-fast-math", "-ffp-contract=off", "-fopenmp", "-fPIC",
+               "-shared", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.skim_oracle_row_stride_words.restype = C.c_int64
+        _lib.skim_oracle_row_stride_words.argtypes = [C.c_int64, C.c_int]
+        _lib.skim_oracle_float_to_half.restype = C.c_uint16
+        _lib.skim_oracle_float_to_half.argtypes = [C.c_float]
+        _lib.skim_oracle_half_to_float.restype = C.c_float
+        _lib.skim_oracle_half_to_float.argtypes = [C.c_uint16]
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().skim_oracle_num_threads())
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _bit_array(bit_set):
+    arr = np.ascontiguousarray(bit_set, dtype=np.int32)
+    return arr, int(sum(1 << int(b) for b in arr))
+
+
+def kmeans_row(x, g, k, iters, round_fp32=True, want_trace=False):
+    """One row: returns dict(c, label, err, trace, n_distinct)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    m = x.shape[0]
+    c = np.zeros(k, dtype=np.float64)
+    label = np.zeros(m, dtype=np.int32)
+    err = C.c_double(0.0)
+    nd = C.c_int(0)
+    trace = np.zeros(2 * iters + 1, dtype=np.float64) if want_trace else None
+    rc = lib().skim_oracle_kmeans_row(_p(x), _p(g), C.c_int64(m), C.c_int(k), C.c_int(iters),
+                                      C.c_int(1 if round_fp32 else 0), _p(c), _p(label),
+                                      C.byref(err), _p(trace), C.byref(nd))
+    if rc:
+        raise ValueError(f"skim_oracle_kmeans_row failed ({rc})")
+    return dict(c=c, label=label, err=err.value, trace=trace, n_distinct=nd.value)
+
+
+def cluster_rows(W, importance, bit_set, iters, s=None, row_bits=None, round_fp32=True,
+                 want_codes=True, want_trace=False):
+    """All rows at all bit-widths.  ``W`` float16 [rows, cols]; ``importance`` float32.
+
+    Returns dict(centroids float64 [rows, sum 2^b], codes uint8 [n_bits, rows, cols] or None,
+    err float64 [rows, n_bits], trace or None).
+    """
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.float16 and W.ndim == 2
+    importance = np.ascontiguousarray(importance, dtype=np.float32)
+    assert importance.shape == W.shape
+    rows, cols = W.shape
+    bits, sumk = _bit_array(bit_set)
+    nb = len(bits)
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+        assert s.shape == (cols,)
+    if row_bits is not None:
+        row_bits = np.ascontiguousarray(row_bits, dtype=np.uint8)
+    centroids = np.zeros((rows, sumk), dtype=np.float64)
+    codes = np.zeros((nb, rows, cols), dtype=np.uint8) if want_codes else None
+    err = np.zeros((rows, nb), dtype=np.float64)
+    trace = np.zeros((rows, nb, 2 * iters + 1), dtype=np.float64) if want_trace else None
+    rc = lib().skim_oracle_cluster_rows(_p(W.view(np.uint16)), _p(importance), C.c_int64(rows),
+                                        C.c_int64(cols), C.c_int64(cols), _p(s), _p(row_bits),
+                                        _p(bits), C.c_int(nb), C.c_int(iters),
+                                        C.c_int(1 if round_fp32 else 0), _p(centroids), _p(codes),
+                                        _p(err), _p(trace))
+    if rc:
+        raise ValueError(f"skim_oracle_cluster_rows failed ({rc})")
+    return dict(centroids=centroids, codes=codes, err=err, trace=trace)
+
+
+def allocate_bits(err, b_min, budget):
+    """Greedy allocation over a float32 table [rows, n_bits]; returns (bits uint8 [rows], total)."""
+    err = np.ascontiguousarray(err, dtype=np.float32)
+    rows, nb = err.shape
+    bits = np.zeros(rows, dtype=np.uint8)
+    total = C.c_int64(0)
+    rc = lib().skim_oracle_allocate_bits(_p(err), C.c_int64(rows), C.c_int(nb), C.c_int(b_min),
+                                         C.c_double(budget), _p(bits), C.byref(total))
+    if rc == -2:
+        raise ValueError("budget outside [b_min, b_max]")
+    if rc:
+        raise ValueError(f"skim_oracle_allocate_bits failed ({rc})")
+    return bits, total.value
+
+
+def row_stride_words(cols, b):
+    return int(lib().skim_oracle_row_stride_words(C.c_int64(cols), C.c_int(b)))
+
+
+def emit(W, bits, centroids, bit_set, s=None):
+    """Packed codes, row order, group starts/offsets, fp16 LUT and unpacked codes."""
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.float16
+    rows, cols = W.shape
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    centroids = np.ascontiguousarray(centroids, dtype=np.float32)
+    bs, sumk = _bit_array(bit_set)
+    nb = len(bs)
+    assert centroids.shape == (rows, sumk)
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+    kmax = 1 << int(bs[-1])
+    max_words = rows * row_stride_words(cols, int(bs[-1]))
+    packed = np.zeros(max_words, dtype=np.uint32)
+    row_order = np.zeros(rows, dtype=np.int32)
+    group_start = np.zeros(nb + 1, dtype=np.int64)
+    group_word = np.zeros(nb + 1, dtype=np.int64)
+    lut = np.zeros((rows, kmax), dtype=np.uint16)
+    codes = np.zeros((rows, cols), dtype=np.uint8)
+    rc = lib().skim_oracle_emit(_p(W.view(np.uint16)), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols),
+                                _p(s), _p(bits), _p(centroids), _p(bs), C.c_int(nb), _p(packed),
+                                _p(row_order), _p(group_start), _p(group_word), _p(lut), _p(codes))
+    if rc:
+        raise ValueError(f"skim_oracle_emit failed ({rc})")
+    return dict(packed=packed[:int(group_word[-1])], row_order=row_order, group_start=group_start,
+                group_word=group_word, lut=lut, codes=codes)
+
+
+def scale_loss_grad(W, importance, labels, alpha, want_grad=True):
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.float16
+    importance = np.ascontiguousarray(importance, dtype=np.float32)
+    labels = np.ascontiguousarray(labels, dtype=np.uint8)
+    alpha = np.ascontiguousarray(alpha, dtype=np.float64)
+    rows, cols = W.shape
+    loss = C.c_double(0.0)
+    grad = np.zeros(cols, dtype=np.float64) if want_grad else None
+    rc = lib().skim_oracle_scale_loss_grad(_p(W.view(np.uint16)), _p(importance), C.c_int64(rows),
+                                           C.c_int64(cols), C.c_int64(cols), _p(labels), _p(alpha),
+                                           C.byref(loss), _p(grad))
+    if rc:
+        raise ValueError(f"skim_oracle_scale_loss_grad failed ({rc})")
+    return loss.value, grad
+
+
+def scale_update(W, importance, labels, alpha, steps=120, lr0=0.01, decay=0.5, decay_every=40,
+                 beta1=0.9, beta2=0.999, eps=1e-8):
+    """Returns (alpha float64 [cols] after `steps` Adam steps, loss trace [steps])."""
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.float16
+    importance = np.ascontiguousarray(importance, dtype=np.float32)
+    labels = np.ascontiguousarray(labels, dtype=np.uint8)
+    alpha = np.array(alpha, dtype=np.float64, copy=True)
+    rows, cols = W.shape
+    trace = np.zeros(steps, dtype=np.float64)
+    rc = lib().skim_oracle_scale_update(_p(W.view(np.uint16)), _p(importance), C.c_int64(rows),
+                                        C.c_int64(cols), C.c_int64(cols), _p(labels), _p(alpha),
+                                        C.c_int(steps), C.c_double(lr0), C.c_double(decay),
+                                        C.c_int(decay_every), C.c_double(beta1), C.c_double(beta2),
+                                        C.c_double(eps), _p(trace))
+    if rc:
+        raise ValueError(f"skim_oracle_scale_update failed ({rc})")
+    return alpha, trace
