@@ -1,0 +1,190 @@
+/*
+ * skim.h -- C ABI of the B200 (sm_100a) implementation of SKIM's row-clustering path
+ * (SKIM: Scaled K-means clustering wIth Mixed precision, arXiv 2412.04180).
+ *
+ * The calls follow the paper's problem statement (Algorithm 3: inputs W, squared gradients G,
+ * the bit budget and the available widths b_min..b_max; outputs labels L, centroids c, scaling
+ * vector alpha):
+ *
+ *   skim_cluster_rows     error pre-recording: weighted 1-D K-means of every row at every
+ *                         candidate width                      (Algorithm 3, first loop nest)
+ *   skim_allocate_bits    greedy mixed-precision allocation     (Section 4.2, Algorithm 1)
+ *   skim_quantize         labels at the allocated width, packed by width group, and the
+ *                         per-row codebook                      (Algorithm 3, second loop;
+ *                                                                Section 4.2, last paragraph)
+ *   skim_apply_scale      installs the scaling vector alpha: all later calls cluster
+ *                         W * alpha^-1                          (Section 4.3, Algorithm 2)
+ *   skim_cluster_rows_at  re-clustering at the already allocated widths inside the
+ *                         grouping/scaling alternation          (Algorithm 2, outer loop)
+ *   skim_scale_update     Adam steps on alpha with the labels fixed
+ *                                                               (Algorithm 2, inner repeat)
+ *
+ * Conventions
+ *   - Every array argument is a DEVICE pointer owned by the caller unless its comment says
+ *     "host".  The library allocates no device memory: scratch comes from the workspace the
+ *     caller sizes with skim_workspace_bytes and hands over with skim_set_workspace.
+ *   - Work is enqueued on the stream given to skim_create and is asynchronous with respect to
+ *     the host; outputs are valid once that stream has reached the end of the call's work.
+ *   - Every call returns SKIM_OK (0) or a negative SKIM_ERR_* code.  Argument errors are found
+ *     on the host before anything is launched.  Bad data (NaN/Inf weights, negative or NaN
+ *     importance, zero or non-finite scale entries) never faults: it sets bits in a device
+ *     status word that skim_get_status reads back; outputs of affected rows are unspecified.
+ *   - W holds IEEE binary16 bit patterns, row-major, `ld` elements between rows (ld >= cols);
+ *     importance holds binary32 with the same layout.  Rows are output channels.
+ *   - bit_set (host) lists the candidate widths: strictly ascending, consecutive integers,
+ *     all inside [1, SKIM_MAX_BIT].  Width b has 2^b centroids.  "sumk" below is the sum of
+ *     2^b over bit_set; a row's centroid record is the concatenation of its width blocks in
+ *     bit_set order, each block ascending.
+ *   - The value that is clustered is x = float(W_ij) when no scale is installed, else the
+ *     binary32 product float(W_ij) * r_j with r_j = 1.0f / s_j.
+ */
+#ifndef SKIM_H_
+#define SKIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SKIM_OK 0
+#define SKIM_ERR_NULL (-1)        /* a required pointer is NULL */
+#define SKIM_ERR_SHAPE (-2)       /* rows/cols/ld/iters out of range (cols above skim_max_cols included) */
+#define SKIM_ERR_BITSET (-3)      /* bit_set not ascending-consecutive inside [1, SKIM_MAX_BIT] */
+#define SKIM_ERR_BUDGET (-4)      /* budget outside [b_min, b_max] */
+#define SKIM_ERR_WORKSPACE (-5)   /* workspace missing, too small or misaligned */
+#define SKIM_ERR_CUDA (-6)        /* a CUDA runtime call failed */
+#define SKIM_ERR_BAD_DATA (-7)    /* reported by skim_get_status: the status word is non-zero */
+#define SKIM_ERR_SCALE (-8)       /* installed scale vector length differs from cols */
+#define SKIM_ERR_ALIGN (-9)       /* an output pointer is not aligned as documented */
+
+#define SKIM_MAX_BIT 4            /* the paper caps the width at 4 bits (Section 5.1) */
+
+/* status bits */
+#define SKIM_STATUS_BAD_WEIGHT 1ull      /* NaN or Inf in W */
+#define SKIM_STATUS_BAD_IMPORTANCE 2ull  /* NaN, Inf or negative importance */
+#define SKIM_STATUS_BAD_SCALE 4ull       /* zero, negative or non-finite scale entry */
+
+typedef struct skim_ctx skim_ctx;
+
+/* Creates a context bound to `device` and to `cuda_stream` (a cudaStream_t cast to void*; NULL is
+ * the legacy default stream).  The context owns only host memory.  `out` receives it. */
+int skim_create(skim_ctx **out, int device, void *cuda_stream);
+int skim_destroy(skim_ctx *ctx);
+
+/* Largest `cols` the device's shared memory lets one row occupy (22 528 on B200). */
+int skim_max_cols(const skim_ctx *ctx, int64_t *out);
+
+/* Bytes of device scratch needed for matrices of up to rows x cols; `out` is a host pointer.
+ * The workspace must be 256-byte aligned and stays owned by the caller.  It also stores the
+ * installed scale vector, so it must outlive every call that follows skim_apply_scale. */
+int skim_workspace_bytes(int64_t rows, int64_t cols, size_t *out);
+int skim_set_workspace(skim_ctx *ctx, void *workspace, size_t bytes);
+
+/* Section 4.3: installs the scaling vector s = alpha (device, [cols], every entry finite and
+ * > 0), stored as r = 1.0f/s in the workspace; s == NULL removes it (alpha = 1).  The caller's
+ * buffer is not referenced after the call's work has run. */
+int skim_apply_scale(skim_ctx *ctx, const float *s, int64_t cols);
+
+/*
+ * Algorithm 3, error pre-recording.  For every row i and every width b in bit_set: weighted
+ * K-means (objective sum_j g_ij (x_ij - c)^2, Section 3.2 diagonal form) with 2^b centroids,
+ * index-quantile init, exactly `iters` assign/update pairs, one final assignment.
+ *   centroids  out [rows][sumk] binary32; may be NULL
+ *   codes      out [n_bits][rows][cols] uint8 labels of the final assignment; may be NULL
+ *   err        out [rows][n_bits] binary32: the objective at the final assignment
+ * iters >= 0.  1 <= cols <= skim_max_cols.  rows >= 0 (0 is a no-op).
+ */
+int skim_cluster_rows(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
+                      int64_t cols, int64_t ld, const int *bit_set, int n_bits, int iters,
+                      float *centroids, uint8_t *codes, float *err);
+
+/*
+ * Algorithm 2, outer loop (and Algorithm 3, second loop): as skim_cluster_rows, but row i is
+ * clustered only at its allocated width row_bits[i] (device, uint8, a member of bit_set).
+ *   centroids  out [rows][sumk]: only the block of the row's width is written
+ *   codes      out [rows][cols] uint8, may be NULL
+ *   err        out [rows] binary32, may be NULL
+ */
+int skim_cluster_rows_at(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
+                         int64_t cols, int64_t ld, const uint8_t *row_bits, const int *bit_set,
+                         int n_bits, int iters, float *centroids, uint8_t *codes, float *err);
+
+/*
+ * Algorithm 1.  All rows start at b_min; the row with the largest error reduction
+ * err[i][b_i] - err[i][b_i+1] (differences taken in binary64; lowest row index on ties) gains a
+ * bit until the total is T = floor(rows * budget + 1e-6).  Reductions may be negative.
+ *   err         [rows][n_bits] binary32 (column u is width bit_set[u])
+ *   bits        out [rows] uint8
+ *   total_bits  host out, may be NULL: T (computed on the host, no synchronisation)
+ */
+int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
+                       double budget, uint8_t *bits, int64_t *total_bits);
+
+/* Packed layout (host-only helper): 32-bit words per packed row of each width,
+ * ceil(cols*b/32) rounded up to a multiple of 4, and the byte size that is enough for any
+ * allocation (every row at the largest width).  Outputs are host pointers; either may be NULL. */
+int skim_packed_layout(int64_t rows, int64_t cols, const int *bit_set, int n_bits,
+                       int64_t *row_stride_words, size_t *max_packed_bytes);
+
+/*
+ * Algorithm 3, final labels and codebooks, packed as Section 4.2 describes: rows of equal width
+ * are gathered (ascending width, ascending row index inside a group) and stored back to back.
+ *   bits        [rows] uint8 allocated widths
+ *   centroids   [rows][sumk] binary32 (from skim_cluster_rows or skim_cluster_rows_at)
+ *   packed      out, 16-byte aligned: a packed row is a little-endian bit stream, element j in
+ *               bits [j*b, (j+1)*b) of the row, zero padded to the row stride
+ *   row_order   out [rows] int32: source row of every packed row
+ *   group_info  out [2*(n_bits+1)] int64: first packed row of every width group, then the
+ *               32-bit-word offset of every group inside `packed` (last entries: totals)
+ *   lut         out [rows][2^b_max] binary16 bit patterns of the row's centroids, round to
+ *               nearest even, entries beyond 2^b_i repeat the last one
+ * The label of an element is the number of midpoints (c_j + c_{j+1})/2 that lie strictly below it.
+ */
+int skim_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
+                  const uint8_t *bits, const float *centroids, const int *bit_set, int n_bits,
+                  uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);
+
+/*
+ * Algorithm 2, inner repeat: `steps` Adam updates (Section 5.1: learning rate lr0, multiplied
+ * by `decay` every `decay_every` steps; betas 0.9/0.999, eps 1e-8) of the scaling vector with the
+ * labels fixed, on loss = sum g_ij (W_ij - alpha_j c_{i,l_ij})^2 with importance-weighted
+ * centroids c of W * alpha^-1 re-fitted at every step.
+ *   labels      [rows][cols] uint8 (as written by skim_cluster_rows_at)
+ *   alpha       in/out [cols] binary32, every entry > 0
+ *   loss_trace  out, may be NULL: [steps] binary64, the loss at the alpha each step started from
+ * Does not install alpha; call skim_apply_scale(alpha) afterwards to cluster with it.
+ */
+int skim_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
+                      int64_t cols, int64_t ld, const uint8_t *labels, float *alpha, int steps,
+                      float lr0, float decay, int decay_every, double *loss_trace);
+
+/*
+ * The whole path from HOST buffers: copies W and importance to the device staging area, runs
+ * skim_cluster_rows, skim_allocate_bits and skim_quantize, and copies the results back, then
+ * waits for the stream.  `staging` is device memory of at least skim_host_staging_bytes bytes,
+ * 256-byte aligned.  Host outputs (any may be NULL): err [rows][n_bits], bits [rows], packed
+ * (skim_packed_layout max bytes), row_order [rows], group_info [2*(n_bits+1)],
+ * lut [rows][2^b_max].
+ */
+int skim_host_staging_bytes(int64_t rows, int64_t cols, const int *bit_set, int n_bits, size_t *out);
+int skim_quantize_matrix_host(skim_ctx *ctx, const uint16_t *W_host, const float *importance_host,
+                              int64_t rows, int64_t cols, const int *bit_set, int n_bits, int iters,
+                              double budget, void *staging, size_t staging_bytes, float *err_host,
+                              uint8_t *bits_host, uint32_t *packed_host, int32_t *row_order_host,
+                              int64_t *group_info_host, uint16_t *lut_host);
+
+/* Reads and clears the device status word (synchronises the stream).  Returns SKIM_OK when it
+ * was zero, SKIM_ERR_BAD_DATA otherwise; `flags` (host, may be NULL) receives the bits. */
+int skim_get_status(skim_ctx *ctx, uint64_t *flags);
+
+/* Number of kernel launches the context has issued so far (host counter). */
+int64_t skim_launch_count(const skim_ctx *ctx);
+
+const char *skim_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKIM_H_ */
