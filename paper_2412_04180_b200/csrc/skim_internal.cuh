@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of libskim.so.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "skim.h"
+
+#define SKIM_MAX_NBITS SKIM_MAX_BIT
+#define SKIM_MAX_SUMK 30  // 2 + 4 + 8 + 16: one warp lane per centroid
+
+struct skim_ctx {
+    int device;
+    cudaStream_t stream;
+    int sm_count;
+    int max_smem_optin;   // bytes of dynamic shared memory one block may opt into
+    void *ws;             // caller's workspace
+    size_t ws_bytes;
+    bool scaled;          // a scale vector is installed
+    int64_t scale_cols;
+    int64_t launches;
+};
+
+// Workspace layout (all offsets 256-byte aligned), carved per call for the call's (rows, cols).
+// The status word and the reciprocal scale sit at fixed offsets, so they persist across calls.
+struct SkimWorkspace {
+    unsigned long long *status;  // 1 word
+    float *rscale;               // [cols]     reciprocal of the installed scale vector
+    int32_t *row_pos;            // [rows]     packed-row index of every source row
+    double *alpha64;             // [cols]     scale-update master copy of alpha
+    double *adam_m;              // [cols]
+    double *adam_v;              // [cols]
+    double *ralpha;              // [cols]     1 / alpha (binary64)
+    double *loss_part;           // [SKIM_SCALE_MAX_CTAS]
+    double *grad_part;           // [SKIM_SCALE_MAX_CTAS][cols]
+    size_t bytes;
+};
+
+#define SKIM_SCALE_MAX_CTAS 296
+
+static inline size_t skim_align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+static inline SkimWorkspace skim_carve(void *base, int64_t rows, int64_t cols)
+{
+    SkimWorkspace w;
+    char *p = (char *)base;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char *q = p ? p + off : nullptr; off += skim_align256(bytes); return q; };
+    w.status = (unsigned long long *)take(256);
+    w.rscale = (float *)take((size_t)cols * 4);
+    w.row_pos = (int32_t *)take((size_t)rows * 4);
+    w.alpha64 = (double *)take((size_t)cols * 8);
+    w.adam_m = (double *)take((size_t)cols * 8);
+    w.adam_v = (double *)take((size_t)cols * 8);
+    w.ralpha = (double *)take((size_t)cols * 8);
+    w.loss_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * 8);
+    w.grad_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * (size_t)cols * 8);
+    w.bytes = off;
+    return w;
+}
+
+// Validated description of a bit set.
+struct SkimBits {
+    int n_bits;
+    int b_min;
+    int b_max;
+    int sumk;
+};
+
+int skim_check_bits(const int *bit_set, int n_bits, SkimBits *out);
+
+#define SKIM_CUDA_OK(expr)                         \
+    do {                                           \
+        cudaError_t e_ = (expr);                   \
+        if (e_ != cudaSuccess) return SKIM_ERR_CUDA; \
+    } while (0)
+
+// Launchers implemented in the kernel translation units.  All return SKIM_OK or SKIM_ERR_*.
+int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
+                        int64_t cols, int64_t ld, const uint8_t *row_bits, const SkimBits &bits,
+                        int iters, float *centroids, uint8_t *codes, float *err);
+int skim_cluster_max_cols(int max_smem_optin, int64_t *out);
+int skim_launch_reciprocal(skim_ctx *ctx, const float *s, int64_t cols);
+int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits,
+                         int64_t K, uint8_t *out_bits);
+int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
+                         const uint8_t *bits, const float *centroids, const SkimBits &bs,
+                         uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);
+int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
+                             int64_t cols, int64_t ld, const uint8_t *labels, float *alpha, int steps,
+                             float lr0, float decay, int decay_every, double *loss_trace);
+
+__host__ __device__ static inline int64_t skim_row_stride_words(int64_t cols, int b)
+{
+    int64_t w = (cols * (int64_t)b + 31) / 32;
+    return (w + 3) / 4 * 4;
+}

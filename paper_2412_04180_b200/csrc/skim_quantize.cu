@@ -1,0 +1,247 @@
+// Final labels, packing and codebooks (SKIM Algorithm 3, second row loop; Section 4.2: rows of
+// equal width are gathered and packed together), plus the reciprocal of the scaling vector
+// (Section 4.3).
+//
+//   skim_rank_rows_kernel  one block: stable partition of the rows by width -> packed position of
+//                          every row, row order, group starts and word offsets.
+//   skim_pack_kernel       one block per row: label = number of midpoints below the element
+//                          (4-step search over <= 15 boundaries), 8 labels per thread, four
+//                          threads merge their bit fields with shuffles and store whole words.
+#include "skim_internal.cuh"
+
+namespace {
+
+constexpr int RT = 1024;
+
+__global__ void __launch_bounds__(RT) skim_rank_rows_kernel(const uint8_t *__restrict__ bits, int64_t n, int64_t cols,
+                                                             int nb, int bmin, int32_t *__restrict__ row_pos,
+                                                             int32_t *__restrict__ row_order,
+                                                             long long *__restrict__ group_info,
+                                                             unsigned long long *status)
+{
+    __shared__ int wsum[RT / 32][SKIM_MAX_NBITS];
+    __shared__ int gstart[SKIM_MAX_NBITS + 1];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t per = (n + RT - 1) / RT;
+    const int64_t r0 = min(n, (int64_t)tid * per), r1 = min(n, r0 + per);
+    int cnt[SKIM_MAX_NBITS] = {0, 0, 0, 0};
+    bool bad = false;
+    for (int64_t i = r0; i < r1; ++i) {
+        const int u = (int)bits[i] - bmin;
+        if (u < 0 || u >= nb) { bad = true; continue; }
+#pragma unroll
+        for (int v = 0; v < SKIM_MAX_NBITS; ++v) cnt[v] += (u == v) ? 1 : 0;
+    }
+    if (bad) atomicOr(status, 8ull);
+    int inc[SKIM_MAX_NBITS];
+#pragma unroll
+    for (int v = 0; v < SKIM_MAX_NBITS; ++v) inc[v] = cnt[v];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+#pragma unroll
+        for (int v = 0; v < SKIM_MAX_NBITS; ++v) {
+            const int t = __shfl_up_sync(0xffffffffu, inc[v], off);
+            if (lane >= off) inc[v] += t;
+        }
+    }
+    if (lane == 31) {
+#pragma unroll
+        for (int v = 0; v < SKIM_MAX_NBITS; ++v) wsum[warp][v] = inc[v];
+    }
+    __syncthreads();
+    int before[SKIM_MAX_NBITS], total[SKIM_MAX_NBITS];
+#pragma unroll
+    for (int v = 0; v < SKIM_MAX_NBITS; ++v) {
+        before[v] = inc[v] - cnt[v];
+        total[v] = 0;
+        for (int w = 0; w < RT / 32; ++w) {
+            const int s = wsum[w][v];
+            if (w < warp) before[v] += s;
+            total[v] += s;
+        }
+    }
+    if (tid == 0) {
+        long long start = 0, word = 0;
+        for (int v = 0; v < nb; ++v) {
+            gstart[v] = (int)start;
+            group_info[v] = start;
+            group_info[nb + 1 + v] = word;
+            start += total[v];
+            word += (long long)total[v] * skim_row_stride_words(cols, bmin + v);
+        }
+        gstart[nb] = (int)start;
+        group_info[nb] = start;
+        group_info[2 * nb + 1] = word;
+    }
+    __syncthreads();
+    for (int64_t i = r0; i < r1; ++i) {
+        const int u = (int)bits[i] - bmin;
+        if (u < 0 || u >= nb) { row_pos[i] = -1; continue; }
+        int pos = 0;
+#pragma unroll
+        for (int v = 0; v < SKIM_MAX_NBITS; ++v) {
+            if (u == v) { pos = gstart[v] + before[v]; before[v] += 1; }
+        }
+        row_pos[i] = pos;
+        row_order[pos] = (int32_t)i;
+    }
+}
+
+constexpr int PT = 256;
+
+struct PackArgs {
+    const uint16_t *W;
+    const float *rscale;
+    const uint8_t *bits;
+    const float *centroids;
+    const int32_t *row_pos;
+    const long long *group_info;
+    int64_t ld;
+    int cols;
+    int nb, bmin, sumk;
+    int vec_ok;   // rows start 16-byte aligned: 128-bit loads allowed
+    uint32_t *packed;
+    uint16_t *lut;
+};
+
+__global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
+{
+    __shared__ float tf[16];
+    const int tid = threadIdx.x;
+    const int64_t row = blockIdx.x;
+    const int pos = a.row_pos[row];
+    if (pos < 0) return;
+    const int b = (int)a.bits[row];
+    const int bi = b - a.bmin;
+    const int k = 1 << b;
+    const int off = (1 << a.bmin) * ((1 << bi) - 1);
+    const int kmax = 1 << (a.bmin + a.nb - 1);
+    const float *c = a.centroids + row * a.sumk + off;
+    if (tid < 16) {
+        const float cj = c[min(tid, k - 1)];
+        if (tid < kmax) a.lut[row * kmax + tid] = __half_as_ushort(__float2half_rn(cj));
+        float t = __int_as_float(0x7f800000);
+        if (tid < k - 1) {
+            t = __double2float_rd(0.5 * ((double)cj + (double)c[tid + 1]));
+            if (t == 0.0f) t = 0.0f;
+        }
+        tf[tid] = t;
+    }
+    __syncthreads();
+    const int64_t stride = skim_row_stride_words(a.cols, b);
+    uint32_t *dst = a.packed + a.group_info[a.nb + 1 + bi] + (int64_t)(pos - a.group_info[bi]) * stride;
+    const int ngroups = (int)((stride + b - 1) / b);   // a group: 32 elements -> b words
+    const uint16_t *Wr = a.W + row * a.ld;
+    const int quad = tid >> 2, ql = tid & 3;
+    for (int base = 0; base < ngroups; base += PT / 4) {
+        const int grp = base + quad;
+        const int e0 = grp * 32 + ql * 8;
+        float x[8];
+        if (a.vec_ok && e0 + 8 <= a.cols) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(Wr + e0);
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float2 f = __half22float2(h2[u]);
+                x[2 * u] = f.x;
+                x[2 * u + 1] = f.y;
+            }
+            if (a.rscale) {
+                const float4 r0 = *reinterpret_cast<const float4 *>(a.rscale + e0);
+                const float4 r1 = *reinterpret_cast<const float4 *>(a.rscale + e0 + 4);
+                x[0] = __fmul_rn(x[0], r0.x); x[1] = __fmul_rn(x[1], r0.y);
+                x[2] = __fmul_rn(x[2], r0.z); x[3] = __fmul_rn(x[3], r0.w);
+                x[4] = __fmul_rn(x[4], r1.x); x[5] = __fmul_rn(x[5], r1.y);
+                x[6] = __fmul_rn(x[6], r1.z); x[7] = __fmul_rn(x[7], r1.w);
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int e = e0 + u;
+                float v = -__int_as_float(0x7f800000);    // past the row: label 0 (zero padding)
+                if (e < a.cols) {
+                    v = __half2float(__ushort_as_half(Wr[e]));
+                    if (a.rscale) v = __fmul_rn(v, a.rscale[e]);
+                }
+                x[u] = v;
+            }
+        }
+        uint32_t v = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int code = (x[u] > tf[7]) ? 8 : 0;
+            code += (x[u] > tf[code + 3]) ? 4 : 0;
+            code += (x[u] > tf[code + 1]) ? 2 : 0;
+            code += (x[u] > tf[code]) ? 1 : 0;
+            v |= (uint32_t)code << (u * b);
+        }
+        const int sh = ql * 8 * b;                           // bit offset inside the group's b words
+        unsigned long long lo = 0ull, hi = 0ull;
+        if (sh < 64) {
+            lo = (unsigned long long)v << sh;
+            if (sh + 8 * b > 64) hi = (unsigned long long)v >> (64 - sh);
+        } else {
+            hi = (unsigned long long)v << (sh - 64);
+        }
+        lo |= __shfl_xor_sync(0xffffffffu, lo, 1);
+        hi |= __shfl_xor_sync(0xffffffffu, hi, 1);
+        lo |= __shfl_xor_sync(0xffffffffu, lo, 2);
+        hi |= __shfl_xor_sync(0xffffffffu, hi, 2);
+        const unsigned long long half = (ql < 2) ? lo : hi;
+        const uint32_t word = (uint32_t)(half >> (32 * (ql & 1)));
+        const int64_t widx = (int64_t)grp * b + ql;
+        if (grp < ngroups && ql < b && widx < stride) dst[widx] = word;
+    }
+}
+
+__global__ void skim_reciprocal_kernel(const float *__restrict__ s, int64_t cols, float *__restrict__ r,
+                                       unsigned long long *status)
+{
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= cols) return;
+    const float v = s[j];
+    if (!(v > 0.0f) || v > 3.0e38f) atomicOr(status, (unsigned long long)SKIM_STATUS_BAD_SCALE);
+    r[j] = __fdiv_rn(1.0f, v);
+}
+
+}  // namespace
+
+int skim_launch_reciprocal(skim_ctx *ctx, const float *s, int64_t cols)
+{
+    SkimWorkspace ws = skim_carve(ctx->ws, 0, cols);
+    const int threads = 256;
+    const unsigned blocks = (unsigned)((cols + threads - 1) / threads);
+    skim_reciprocal_kernel<<<blocks, threads, 0, ctx->stream>>>(s, cols, ws.rscale, ws.status);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    return SKIM_OK;
+}
+
+int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
+                         const uint8_t *bits, const float *centroids, const SkimBits &bs, uint32_t *packed,
+                         int32_t *row_order, int64_t *group_info, uint16_t *lut)
+{
+    SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
+    skim_rank_rows_kernel<<<1, RT, 0, ctx->stream>>>(bits, rows, cols, bs.n_bits, bs.b_min, ws.row_pos, row_order,
+                                                     (long long *)group_info, ws.status);
+    SKIM_CUDA_OK(cudaGetLastError());
+    PackArgs a;
+    a.W = W;
+    a.rscale = ctx->scaled ? ws.rscale : nullptr;
+    a.bits = bits;
+    a.centroids = centroids;
+    a.row_pos = ws.row_pos;
+    a.group_info = (const long long *)group_info;
+    a.ld = ld;
+    a.cols = (int)cols;
+    a.nb = bs.n_bits;
+    a.bmin = bs.b_min;
+    a.sumk = bs.sumk;
+    a.vec_ok = ((reinterpret_cast<uintptr_t>(W) & 15u) == 0 && (ld % 8) == 0) ? 1 : 0;
+    a.packed = packed;
+    a.lut = lut;
+    skim_pack_kernel<<<(unsigned)rows, PT, 0, ctx->stream>>>(a);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 2;
+    return SKIM_OK;
+}

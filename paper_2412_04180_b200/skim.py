@@ -1,0 +1,253 @@
+"""Thin Python binding of libskim.so (argument marshalling only; every step runs in the CUDA
+kernels behind the C ABI declared in ``include/skim.h``).
+
+PyTorch is used for device memory and streams.  There is no CPU fallback: loading fails
+loudly when the library has not been built, and every call needs CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libskim.so")
+_lib = None
+
+ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_ERR_BITSET",
+             -4: "SKIM_ERR_BUDGET", -5: "SKIM_ERR_WORKSPACE", -6: "SKIM_ERR_CUDA",
+             -7: "SKIM_ERR_BAD_DATA", -8: "SKIM_ERR_SCALE", -9: "SKIM_ERR_ALIGN"}
+
+EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
+           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits",
+           "skim_packed_layout", "skim_quantize", "skim_scale_update", "skim_host_staging_bytes",
+           "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_strerror"]
+
+
+class SkimError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = lib().skim_strerror(code).decode()
+        super().__init__(f"{where}: {ERR_NAMES.get(code, code)} ({msg})")
+
+
+def lib():
+    """Loads libskim.so; raises if it is missing (build it with ``python -m paper_2412_04180_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: the CUDA library has not been built "
+                               "(run `python -m paper_2412_04180_b200.build`); there is no fallback")
+        _lib = C.CDLL(LIB_PATH)
+        _lib.skim_strerror.restype = C.c_char_p
+        _lib.skim_strerror.argtypes = [C.c_int]
+        _lib.skim_launch_count.restype = C.c_int64
+        _lib.skim_launch_count.argtypes = [C.c_void_p]
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return C.c_void_p(0)
+    return C.c_void_p(t.data_ptr())
+
+
+def _bits(bit_set):
+    arr = (C.c_int * len(bit_set))(*[int(b) for b in bit_set])
+    return arr, len(bit_set), sum(1 << int(b) for b in bit_set)
+
+
+def _chk(rc, where):
+    if rc != 0:
+        raise SkimError(rc, where)
+
+
+def _dev(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    return t
+
+
+class Skim:
+    """One context: a device, a stream and a caller-owned workspace."""
+
+    def __init__(self, device=0, stream=None, rows=0, cols=0):
+        self.device = torch.device("cuda", device)
+        self._stream = stream
+        handle = C.c_void_p()
+        sp = C.c_void_p(stream.cuda_stream if stream is not None else 0)
+        _chk(lib().skim_create(C.byref(handle), C.c_int(device), sp), "skim_create")
+        self._h = handle
+        self._ws = None
+        if rows and cols:
+            self.reserve(rows, cols)
+
+    def close(self):
+        if self._h is not None:
+            lib().skim_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- workspace
+    def max_cols(self):
+        out = C.c_int64()
+        _chk(lib().skim_max_cols(self._h, C.byref(out)), "skim_max_cols")
+        return out.value
+
+    @staticmethod
+    def workspace_bytes(rows, cols):
+        out = C.c_size_t()
+        _chk(lib().skim_workspace_bytes(C.c_int64(rows), C.c_int64(cols), C.byref(out)), "skim_workspace_bytes")
+        return out.value
+
+    def reserve(self, rows, cols):
+        """Allocates (with torch) and installs a workspace big enough for rows x cols."""
+        nbytes = self.workspace_bytes(rows, cols)
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            self.set_workspace(self._ws)
+
+    def set_workspace(self, buf):
+        _dev(buf, torch.uint8, "workspace")
+        _chk(lib().skim_set_workspace(self._h, _ptr(buf), C.c_size_t(buf.numel())), "skim_set_workspace")
+        self._ws = buf
+
+    # ---- the path
+    def apply_scale(self, s, cols=None):
+        if s is None:
+            _chk(lib().skim_apply_scale(self._h, C.c_void_p(0), C.c_int64(0)), "skim_apply_scale")
+            return
+        _dev(s, torch.float32, "s")
+        _chk(lib().skim_apply_scale(self._h, _ptr(s), C.c_int64(s.numel() if cols is None else cols)),
+             "skim_apply_scale")
+
+    def cluster_rows(self, W, importance, bit_set, iters, want_centroids=True, want_codes=False, ld=None,
+                     cols=None):
+        """Returns (centroids [rows, sumk] or None, codes [n_bits, rows, cols] or None, err [rows, n_bits])."""
+        _dev(W, torch.float16, "W")
+        _dev(importance, torch.float32, "importance")
+        rows = W.shape[0]
+        ld = W.shape[1] if ld is None else ld
+        cols = W.shape[1] if cols is None else cols
+        arr, nb, sumk = _bits(bit_set)
+        cent = torch.empty((rows, sumk), dtype=torch.float32, device=W.device) if want_centroids else None
+        codes = torch.empty((nb, rows, cols), dtype=torch.uint8, device=W.device) if want_codes else None
+        err = torch.empty((rows, nb), dtype=torch.float32, device=W.device)
+        _chk(lib().skim_cluster_rows(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
+                                     C.c_int64(ld), arr, C.c_int(nb), C.c_int(iters), _ptr(cent), _ptr(codes),
+                                     _ptr(err)), "skim_cluster_rows")
+        return cent, codes, err
+
+    def cluster_rows_into(self, W, importance, bit_set, iters, centroids, err, codes=None):
+        """As cluster_rows, writing into caller-provided tensors (no allocation; used when timing)."""
+        rows, cols = W.shape
+        arr, nb, _ = _bits(bit_set)
+        _chk(lib().skim_cluster_rows(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
+                                     C.c_int64(cols), arr, C.c_int(nb), C.c_int(iters), _ptr(centroids),
+                                     _ptr(codes), _ptr(err)), "skim_cluster_rows")
+
+    def cluster_rows_at(self, W, importance, row_bits, bit_set, iters, want_codes=True, centroids=None):
+        """Returns (centroids [rows, sumk], codes [rows, cols] or None, err [rows])."""
+        _dev(W, torch.float16, "W")
+        _dev(importance, torch.float32, "importance")
+        _dev(row_bits, torch.uint8, "row_bits")
+        rows, cols = W.shape
+        arr, nb, sumk = _bits(bit_set)
+        cent = centroids if centroids is not None else torch.zeros((rows, sumk), dtype=torch.float32, device=W.device)
+        codes = torch.empty((rows, cols), dtype=torch.uint8, device=W.device) if want_codes else None
+        err = torch.empty((rows,), dtype=torch.float32, device=W.device)
+        _chk(lib().skim_cluster_rows_at(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
+                                        C.c_int64(cols), _ptr(row_bits), arr, C.c_int(nb), C.c_int(iters),
+                                        _ptr(cent), _ptr(codes), _ptr(err)), "skim_cluster_rows_at")
+        return cent, codes, err
+
+    def allocate_bits(self, err, bit_set, budget, out=None):
+        """Returns (bits uint8 [rows], total_bits)."""
+        _dev(err, torch.float32, "err")
+        rows = err.shape[0]
+        arr, nb, _ = _bits(bit_set)
+        bits = out if out is not None else torch.empty((rows,), dtype=torch.uint8, device=err.device)
+        total = C.c_int64()
+        _chk(lib().skim_allocate_bits(self._h, _ptr(err), C.c_int64(rows), arr, C.c_int(nb), C.c_double(budget),
+                                      _ptr(bits), C.byref(total)), "skim_allocate_bits")
+        return bits, total.value
+
+    @staticmethod
+    def packed_layout(rows, cols, bit_set):
+        """Returns (row stride in 32-bit words for every width, max packed bytes)."""
+        arr, nb, _ = _bits(bit_set)
+        strides = (C.c_int64 * nb)()
+        mx = C.c_size_t()
+        _chk(lib().skim_packed_layout(C.c_int64(rows), C.c_int64(cols), arr, C.c_int(nb), strides, C.byref(mx)),
+             "skim_packed_layout")
+        return list(strides), mx.value
+
+    def quantize(self, W, bits, centroids, bit_set, out=None):
+        """Returns dict(packed uint32 (max size), row_order int32 [rows], group_info int64 [2*(n_bits+1)],
+        lut uint16 [rows, 2^b_max])."""
+        _dev(W, torch.float16, "W")
+        _dev(bits, torch.uint8, "bits")
+        _dev(centroids, torch.float32, "centroids")
+        rows, cols = W.shape
+        arr, nb, _ = _bits(bit_set)
+        if out is None:
+            _, mx = self.packed_layout(rows, cols, bit_set)
+            out = dict(packed=torch.empty(mx // 4, dtype=torch.int32, device=W.device),
+                       row_order=torch.empty(rows, dtype=torch.int32, device=W.device),
+                       group_info=torch.empty(2 * (nb + 1), dtype=torch.int64, device=W.device),
+                       lut=torch.empty((rows, 1 << int(bit_set[-1])), dtype=torch.int16, device=W.device))
+        _chk(lib().skim_quantize(self._h, _ptr(W), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols), _ptr(bits),
+                                 _ptr(centroids), arr, C.c_int(nb), _ptr(out["packed"]), _ptr(out["row_order"]),
+                                 _ptr(out["group_info"]), _ptr(out["lut"])), "skim_quantize")
+        return out
+
+    def scale_update(self, W, importance, labels, alpha, steps=120, lr0=0.01, decay=0.5, decay_every=40,
+                     want_trace=True):
+        """Updates alpha (float32 CUDA tensor) in place; returns the loss trace (float64 [steps]) or None."""
+        _dev(W, torch.float16, "W")
+        _dev(importance, torch.float32, "importance")
+        _dev(labels, torch.uint8, "labels")
+        _dev(alpha, torch.float32, "alpha")
+        rows, cols = W.shape
+        trace = torch.zeros(max(steps, 1), dtype=torch.float64, device=W.device) if want_trace else None
+        _chk(lib().skim_scale_update(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
+                                     C.c_int64(cols), _ptr(labels), _ptr(alpha), C.c_int(steps), C.c_float(lr0),
+                                     C.c_float(decay), C.c_int(decay_every), _ptr(trace)), "skim_scale_update")
+        return trace[:steps] if want_trace else None
+
+    @staticmethod
+    def host_staging_bytes(rows, cols, bit_set):
+        arr, nb, _ = _bits(bit_set)
+        out = C.c_size_t()
+        _chk(lib().skim_host_staging_bytes(C.c_int64(rows), C.c_int64(cols), arr, C.c_int(nb), C.byref(out)),
+             "skim_host_staging_bytes")
+        return out.value
+
+    def quantize_matrix_host(self, W_host, importance_host, bit_set, iters, budget, staging, out):
+        """Whole path from pinned host tensors; ``out`` holds pinned host tensors err, bits, packed,
+        row_order, group_info, lut (any may be missing)."""
+        rows, cols = W_host.shape
+        arr, nb, _ = _bits(bit_set)
+        g = lambda k: _ptr(out.get(k))
+        _chk(lib().skim_quantize_matrix_host(self._h, _ptr(W_host), _ptr(importance_host), C.c_int64(rows),
+                                             C.c_int64(cols), arr, C.c_int(nb), C.c_int(iters), C.c_double(budget),
+                                             _ptr(staging), C.c_size_t(staging.numel()), g("err"), g("bits"),
+                                             g("packed"), g("row_order"), g("group_info"), g("lut")),
+             "skim_quantize_matrix_host")
+
+    def get_status(self):
+        """Returns the status flags (and clears them); 0 means no bad data was seen."""
+        flags = C.c_uint64()
+        rc = lib().skim_get_status(self._h, C.byref(flags))
+        if rc not in (0, -7):
+            raise SkimError(rc, "skim_get_status")
+        return flags.value
+
+    def launch_count(self):
+        return int(lib().skim_launch_count(self._h))
