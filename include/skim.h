@@ -58,6 +58,7 @@ extern "C" {
 #define SKIM_ERR_BAD_DATA (-7)    /* reported by skim_get_status: the status word is non-zero */
 #define SKIM_ERR_SCALE (-8)       /* installed scale vector length differs from cols */
 #define SKIM_ERR_ALIGN (-9)       /* an output pointer is not aligned as documented */
+#define SKIM_ERR_STATIC_LIMIT (-10) /* skim_quantize_static: rows above SKIM_STATIC_MAX_ROWS */
 
 #define SKIM_MAX_BIT 4            /* the paper caps the width at 4 bits (Section 5.1) */
 
@@ -146,6 +147,36 @@ int skim_packed_layout(int64_t rows, int64_t cols, const int *bit_set, int n_bit
 int skim_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
                   const uint8_t *bits, const float *centroids, const int *bit_set, int n_bits,
                   uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);
+
+/*
+ * skim_quantize for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this call; it exists for integration reasons only.)
+ *
+ * Some users of this library run where cudaMalloc is off limits: inside another framework's
+ * allocator or plugin callback, in a process whose device memory was planned and handed out in
+ * full at start-up, or in a latency-critical loop where an allocation's implicit device
+ * synchronisation is not acceptable.  They can neither create a workspace nor let a library do
+ * it.  This variant needs no context and no workspace: the scratch that skim_quantize keeps in
+ * the workspace (one packed-row index per row and a status word) lives in a fixed array inside
+ * the library image, 256 + 4 * SKIM_STATIC_MAX_ROWS bytes on every GPU that loads the library,
+ * held until the process exits.  It calls no cudaMalloc/cudaFree and no allocating routine.
+ *
+ *   - Same inputs, outputs, layout and labels as skim_quantize with no scale vector installed
+ *     (alpha = 1); all array arguments are device pointers, bit_set is a host pointer.
+ *   - Runs on the CURRENT device, on `cuda_stream` (a cudaStream_t cast to void*).
+ *   - rows must not exceed SKIM_STATIC_MAX_ROWS, else SKIM_ERR_STATIC_LIMIT and nothing runs.
+ *   - The first call on a device looks up the array's device address (one
+ *     cudaGetSymbolAddress, cached per device); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents
+ *     (the call clears what it needs at zero).  Two calls that overlap on the GPU -- different
+ *     streams, or different host threads -- race on it: serialise them.
+ *   - A width outside bit_set is skipped, as in skim_quantize; it shows as
+ *     group_info[n_bits] < rows (there is no context to read a status word from).
+ */
+#define SKIM_STATIC_MAX_ROWS 65536
+int skim_quantize_static(void *cuda_stream, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
+                         const uint8_t *bits, const float *centroids, const int *bit_set, int n_bits,
+                         uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);
 
 /*
  * Algorithm 2, inner repeat: `steps` Adam updates (Section 5.1: learning rate lr0, multiplied

@@ -358,6 +358,7 @@ const char *skim_strerror(int code)
     case SKIM_ERR_BAD_DATA: return "bad data: NaN/Inf weight, negative importance, non-positive scale or width outside bit_set";
     case SKIM_ERR_SCALE: return "installed scale vector length differs from cols";
     case SKIM_ERR_ALIGN: return "output pointer not aligned as documented";
+    case SKIM_ERR_STATIC_LIMIT: return "skim_quantize_static: rows exceed SKIM_STATIC_MAX_ROWS (65536), the size of the built-in scratch array";
     default: return "unknown error";
     }
 }

@@ -245,3 +245,84 @@ int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t
     ctx->launches += 2;
     return SKIM_OK;
 }
+
+// ---------------------------------------------------------------- entry point that allocates nothing
+//
+// skim_quantize_static is skim_quantize for callers that cannot provide a workspace because they
+// may not allocate device memory at all: code running inside a region where cudaMalloc is
+// forbidden or would deadlock (an allocator callback, a real-time loop with a fixed memory plan,
+// a plugin that only borrows its host's buffers).  Its scratch (the per-row packed position and a
+// status word) lives in a fixed array inside the library image instead of a caller workspace.
+
+#include <mutex>
+
+#define SKIM_STATIC_SCRATCH_BYTES (256 + (size_t)SKIM_STATIC_MAX_ROWS * 4)
+
+// Resident on every GPU that loads the library, until the process exits.
+static __device__ __align__(256) unsigned char skim_static_scratch[SKIM_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device.  In host code the array's name is
+// only a handle, so the address has to be asked for, once per device, with that device current.
+int static_scratch_address(void **out)
+{
+    int dev = -1;
+    SKIM_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SKIM_ERR_SHAPE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        SKIM_CUDA_OK(cudaGetSymbolAddress(&p, skim_static_scratch));
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return SKIM_OK;
+}
+}  // namespace
+
+extern "C" int skim_quantize_static(void *cuda_stream, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
+                                    const uint8_t *bits, const float *centroids, const int *bit_set, int n_bits,
+                                    uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut)
+{
+    if (!W || !bits || !centroids || !packed || !row_order || !group_info || !lut) return SKIM_ERR_NULL;
+    SkimBits bs;
+    int rc = skim_check_bits(bit_set, n_bits, &bs);
+    if (rc) return rc;
+    if (rows < 1 || cols < 1 || cols > 0x7fffffff / 8 || ld < cols) return SKIM_ERR_SHAPE;
+    if (rows > SKIM_STATIC_MAX_ROWS) return SKIM_ERR_STATIC_LIMIT;
+    if ((reinterpret_cast<uintptr_t>(packed) & 15u) != 0) return SKIM_ERR_ALIGN;
+    void *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long *status = (unsigned long long *)scratch;
+    int32_t *row_pos = (int32_t *)((unsigned char *)scratch + 256);
+    // the array keeps whatever the previous call left: the status word must start at zero
+    // (row_pos is rewritten for every row before it is read)
+    SKIM_CUDA_OK(cudaMemsetAsync(status, 0, 256, stream));
+    skim_rank_rows_kernel<<<1, RT, 0, stream>>>(bits, rows, cols, bs.n_bits, bs.b_min, row_pos, row_order,
+                                                (long long *)group_info, status);
+    SKIM_CUDA_OK(cudaGetLastError());
+    PackArgs a;
+    a.W = W;
+    a.rscale = nullptr;
+    a.bits = bits;
+    a.centroids = centroids;
+    a.row_pos = row_pos;
+    a.group_info = (const long long *)group_info;
+    a.ld = ld;
+    a.cols = (int)cols;
+    a.nb = bs.n_bits;
+    a.bmin = bs.b_min;
+    a.sumk = bs.sumk;
+    a.vec_ok = ((reinterpret_cast<uintptr_t>(W) & 15u) == 0 && (ld % 8) == 0) ? 1 : 0;
+    a.packed = packed;
+    a.lut = lut;
+    skim_pack_kernel<<<(unsigned)rows, PT, 0, stream>>>(a);
+    SKIM_CUDA_OK(cudaGetLastError());
+    return SKIM_OK;
+}

@@ -17,11 +17,11 @@ _lib = None
 
 ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_ERR_BITSET",
              -4: "SKIM_ERR_BUDGET", -5: "SKIM_ERR_WORKSPACE", -6: "SKIM_ERR_CUDA",
-             -7: "SKIM_ERR_BAD_DATA", -8: "SKIM_ERR_SCALE", -9: "SKIM_ERR_ALIGN"}
+             -7: "SKIM_ERR_BAD_DATA", -8: "SKIM_ERR_SCALE", -9: "SKIM_ERR_ALIGN", -10: "SKIM_ERR_STATIC_LIMIT"}
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
            "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits",
-           "skim_packed_layout", "skim_quantize", "skim_scale_update", "skim_host_staging_bytes",
+           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_scale_update", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_strerror"]
 
 
@@ -251,3 +251,28 @@ class Skim:
 
     def launch_count(self):
         return int(lib().skim_launch_count(self._h))
+
+
+STATIC_MAX_ROWS = 65536
+
+
+def quantize_static(W, bits, centroids, bit_set, out, stream=None):
+    """skim_quantize_static: the packer for callers that must not allocate device memory.
+
+    No context and no workspace are involved; the scratch is a fixed array inside the library.
+    ``out`` must hold preallocated CUDA tensors ``packed``, ``row_order``, ``group_info`` and
+    ``lut`` (this wrapper allocates nothing either).  Runs on the current device and on
+    ``stream`` (default: torch's current stream).  Calls that overlap on the GPU race on the
+    shared scratch, so keep them on one stream.
+    """
+    _dev(W, torch.float16, "W")
+    _dev(bits, torch.uint8, "bits")
+    _dev(centroids, torch.float32, "centroids")
+    rows, cols = W.shape
+    arr, nb, _ = _bits(bit_set)
+    st = stream if stream is not None else torch.cuda.current_stream()
+    _chk(lib().skim_quantize_static(C.c_void_p(st.cuda_stream), _ptr(W), C.c_int64(rows), C.c_int64(cols),
+                                    C.c_int64(cols), _ptr(bits), _ptr(centroids), arr, C.c_int(nb),
+                                    _ptr(out["packed"]), _ptr(out["row_order"]), _ptr(out["group_info"]),
+                                    _ptr(out["lut"])), "skim_quantize_static")
+    return out
