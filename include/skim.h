@@ -67,6 +67,7 @@ extern "C" {
 #define SKIM_STATUS_BAD_IMPORTANCE 2ull  /* NaN, Inf or negative importance */
 #define SKIM_STATUS_BAD_SCALE 4ull       /* zero, negative or non-finite scale entry */
 #define SKIM_STATUS_BAD_BITS 8ull        /* an allocated width that is not in bit_set (row skipped) */
+#define SKIM_STATUS_TIMEOUT 16ull        /* an asynchronous copy did not complete within its wait limit (row skipped) */
 
 typedef struct skim_ctx skim_ctx;
 

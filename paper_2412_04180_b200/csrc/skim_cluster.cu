@@ -1,99 +1,31 @@
-// Row clustering kernel: weighted 1-D K-means of one matrix row at every candidate width
+// Generic row-clustering kernel: weighted 1-D K-means of one matrix row at every candidate width
 // (SKIM Algorithm 3, error pre-recording loop; objective of Section 3.2, diagonal form).
+// Handles every case: scaled rows (32-bit keys of the binary32 product) and rows whose layout rules
+// out the vectorised fp16-key kernel of skim_cluster16.cu.
 //
 // One thread block owns one row.
 //   1. load   the row's (value, importance) pairs into registers; the value is turned into an
 //             order-preserving unsigned key.
-//   2. sort   block-wide LSD radix sort (8-bit digits, warp-private digit counters, match-based
+//   2. sort   block-wide LSD radix sort (8-bit digits, warp-private digit counters, ballot-based
 //             stable ranking), exchanging through one shared-memory buffer.  Afterwards every
 //             1-D cluster is a contiguous interval of the sorted row.
-//   3. sums   binary64 prefix sums of g, g*x, g*x^2 at the granularity of small element blocks.
-//   4. Lloyd  one warp, one lane per centroid of every width (2+4+8+16 = 30 lanes).  A lane owns
-//             the boundary between its centroid and the next: the exact midpoint test
-//             x <= (c_j + c_{j+1})/2 becomes an upper-bound search in the sorted keys, interval
-//             sums are differences of prefix sums (plus the ragged ends, summed directly), the
-//             new centroid is the binary64 quotient rounded to binary32.  All widths iterate in
-//             lockstep; the loop ends early once no boundary moved (later iterations would
-//             reproduce the same state exactly).
-//   5. err    sum g (x-c)^2 per interval from the three prefix sums, in binary64.
-#include "skim_internal.cuh"
+//   3.-5.     prefix sums, Lloyd iterations and the error: see skim_cluster_phases.cuh.
+#include "skim_cluster_phases.cuh"
 
 namespace {
+
+using namespace skimk;
 
 constexpr int RADIX_BITS = 8;
 constexpr int RADIX = 1 << RADIX_BITS;
 
-template <typename KeyT> struct KeyOps;
-
-template <> struct KeyOps<uint32_t> {
-    static constexpr int PASSES = 4;
-    static constexpr uint32_t PAD = 0xffffffffu;
-    __device__ static __forceinline__ uint32_t from_float(float x)
-    {
-        uint32_t u = __float_as_uint(x);
-        return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-    }
-    __device__ static __forceinline__ float to_float(uint32_t k)
-    {
-        return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-    }
-    // key of the largest representable value <= t
-    __device__ static __forceinline__ uint32_t floor_key(float t) { return from_float(t); }
-};
-
-template <> struct KeyOps<uint16_t> {
-    static constexpr int PASSES = 2;
-    static constexpr uint16_t PAD = 0xffffu;
-    __device__ static __forceinline__ uint16_t from_half_bits(uint16_t h)
-    {
-        return (h & 0x8000u) ? (uint16_t)~h : (uint16_t)(h | 0x8000u);
-    }
-    __device__ static __forceinline__ float to_float(uint16_t k)
-    {
-        uint16_t h = (k & 0x8000u) ? (uint16_t)(k & 0x7fffu) : (uint16_t)~k;
-        return __half2float(__ushort_as_half(h));
-    }
-    __device__ static __forceinline__ uint16_t floor_key(float t)
-    {
-        uint16_t h = __half_as_ushort(__float2half_rd(t));
-        if (h == 0x8000u) h = 0;
-        return from_half_bits(h);
-    }
-};
-
-struct ClusterArgs {
-    const uint16_t *W;
-    const float *G;
-    const float *rscale;      // nullptr: no scale installed
-    const uint8_t *row_bits;  // nullptr: every width
-    int64_t rows;
-    int64_t ld;
-    int m;                    // cols
-    int nb, bmin, sumk;
-    int iters;
-    int blk_shift;            // log2 of the prefix-sum block length
-    float *centroids;
-    uint8_t *codes;
-    float *err;
-    unsigned long long *status;
-};
-
-struct D3 {
-    double a, b, c;
-};
-
-__device__ __forceinline__ D3 shfl_up3(D3 v, int off)
-{
-    D3 r;
-    r.a = __shfl_up_sync(0xffffffffu, v.a, off);
-    r.b = __shfl_up_sync(0xffffffffu, v.b, off);
-    r.c = __shfl_up_sync(0xffffffffu, v.c, off);
-    return r;
-}
+template <typename KeyT> struct Passes;
+template <> struct Passes<uint32_t> { static constexpr int N = 4; };
+template <> struct Passes<uint16_t> { static constexpr int N = 2; };
 
 // Shared-memory layout, computed identically on host and device.
 struct SmemLayout {
-    size_t keys, gs, uni, wtot, dbase, tfs, dvals, errs, misc, total;
+    size_t keys, gs, uni, dbase, phase, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nwarps, int blk_shift)
@@ -107,12 +39,8 @@ __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nw
     size_t nblk = ((size_t)cap >> blk_shift) + 2;
     size_t prefix = 3 * nblk * 8;
     L.uni = take(counters > prefix ? counters : prefix);
-    L.wtot = take(32 * 3 * 8);
     L.dbase = take(RADIX * 4);
-    L.tfs = take(32 * 4);
-    L.dvals = take(32 * 4);
-    L.errs = take(32 * 8);
-    L.misc = take(64);
+    L.phase = take(sizeof(PhaseSmem));
     L.total = off;
     return L;
 }
@@ -121,6 +49,7 @@ template <typename KeyT, int THREADS, int ITEMS>
 __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
 {
     using K = KeyOps<KeyT>;
+    constexpr int PASSES = Passes<KeyT>::N;
     constexpr int NW = THREADS / 32;
     constexpr int CAP = THREADS * ITEMS;
     extern __shared__ __align__(16) unsigned char smem[];
@@ -129,12 +58,8 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     float *sg = reinterpret_cast<float *>(smem + L.gs);
     uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + L.uni);
     double *PB = reinterpret_cast<double *>(smem + L.uni);
-    double *wtot = reinterpret_cast<double *>(smem + L.wtot);
     uint32_t *dbase = reinterpret_cast<uint32_t *>(smem + L.dbase);
-    float *tfs = reinterpret_cast<float *>(smem + L.tfs);
-    float *dvals = reinterpret_cast<float *>(smem + L.dvals);
-    double *errs = reinterpret_cast<double *>(smem + L.errs);
-    int *misc = reinterpret_cast<int *>(smem + L.misc);   // [0] distinct count, [1] slot counter
+    PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -175,7 +100,7 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     // ---------------------------------------------------------------- 2. sort
     const unsigned lt_mask = (1u << lane) - 1u;
 #pragma unroll 1
-    for (int pass = 0; pass < K::PASSES; ++pass) {
+    for (int pass = 0; pass < PASSES; ++pass) {
         const int shift = pass * RADIX_BITS;
         for (int d = tid; d < NW * RADIX; d += THREADS) cnt[d] = 0;
         __syncthreads();
@@ -217,7 +142,13 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
             const unsigned d = ((unsigned)key[i] >> shift) & (RADIX - 1);
-            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            unsigned peers = 0xffffffffu;   // lanes of this warp whose item has the same digit
+#pragma unroll
+            for (int b = 0; b < RADIX_BITS; ++b) {
+                const bool bit = (d >> b) & 1u;
+                const unsigned bal = __ballot_sync(0xffffffffu, bit);
+                peers &= bit ? bal : ~bal;
+            }
             const uint32_t base = cnt[warp * RADIX + d];
             const unsigned rank = __popc(peers & lt_mask);
             __syncwarp();
@@ -228,7 +159,7 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
             sg[pos] = val[i];
         }
         __syncthreads();
-        if (pass + 1 < K::PASSES) {
+        if (pass + 1 < PASSES) {
 #pragma unroll
             for (int i = 0; i < ITEMS; ++i) {
                 const int e = warp * (ITEMS * 32) + i * 32 + lane;
@@ -240,178 +171,18 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     }
 
     // ---------------------------------------------------------------- 3. distinct count, prefix sums
-    if (tid == 0) { misc[0] = 0; misc[1] = 0; }
+    if (tid == 0) { ps.misc[0] = 0; ps.misc[1] = 0; }
     __syncthreads();
-    {
-        int local = 0;
-        for (int p = tid; p < m; p += THREADS) local += (p == 0 || skeys[p] != skeys[p - 1]) ? 1 : 0;
-#pragma unroll
-        for (int off = 16; off; off >>= 1) local += __shfl_xor_sync(0xffffffffu, local, off);
-        if (lane == 0 && local) atomicAdd(&misc[0], local);
-    }
-    const int BLK = 1 << a.blk_shift;
-    const int nblk = (m + BLK - 1) >> a.blk_shift;
-    double *PB0 = PB, *PB1 = PB + (nblk + 1), *PB2 = PB + 2 * (nblk + 1);
-    {
-        D3 carry = {0.0, 0.0, 0.0};
-        for (int base = 0; base < nblk; base += THREADS) {
-            const int b = base + tid;
-            D3 v = {0.0, 0.0, 0.0};
-            if (b < nblk) {
-                const int lo = b << a.blk_shift;
-                const int hi = min(m, lo + BLK);
-                for (int u = lo; u < hi; ++u) {
-                    const double g = (double)sg[u];
-                    const double x = (double)K::to_float(skeys[u]);
-                    const double gx = g * x;
-                    v.a += g;
-                    v.b += gx;
-                    v.c = fma(gx, x, v.c);
-                }
-            }
-            D3 inc = v;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const D3 t = shfl_up3(inc, off);
-                if (lane >= off) { inc.a += t.a; inc.b += t.b; inc.c += t.c; }
-            }
-            if (lane == 31) { wtot[warp * 3 + 0] = inc.a; wtot[warp * 3 + 1] = inc.b; wtot[warp * 3 + 2] = inc.c; }
-            __syncthreads();
-            D3 wpre = {0.0, 0.0, 0.0}, tot = {0.0, 0.0, 0.0};
-            for (int w = 0; w < NW; ++w) {
-                const double t0 = wtot[w * 3 + 0], t1 = wtot[w * 3 + 1], t2 = wtot[w * 3 + 2];
-                if (w < warp) { wpre.a += t0; wpre.b += t1; wpre.c += t2; }
-                tot.a += t0; tot.b += t1; tot.c += t2;
-            }
-            if (b < nblk) {
-                PB0[b] = carry.a + wpre.a + (inc.a - v.a);
-                PB1[b] = carry.b + wpre.b + (inc.b - v.b);
-                PB2[b] = carry.c + wpre.c + (inc.c - v.c);
-            }
-            carry.a += tot.a; carry.b += tot.b; carry.c += tot.c;
-            __syncthreads();
-        }
-        if (tid == 0) { PB0[nblk] = carry.a; PB1[nblk] = carry.b; PB2[nblk] = carry.c; }
-    }
-    __syncthreads();
-    const int nd = misc[0];   // number of distinct values in the row
-    if (nd <= 16) {
-        // rare: collect the distinct values (ascending) for the widths with 2^b >= nd
-        for (int p = tid; p < m; p += THREADS) {
-            if (p == 0 || skeys[p] != skeys[p - 1]) {
-                const int slot = atomicAdd(&misc[1], 1);
-                if (slot < 16) tfs[slot] = __int_as_float(p);
-            }
-        }
-        __syncthreads();
-        if (warp == 0) {
-            const int p = lane < nd ? __float_as_int(tfs[lane]) : 0x7fffffff;
-            int rank = 0;
-            for (int u = 0; u < nd; ++u) rank += (__shfl_sync(0xffffffffu, p, u) < p) ? 1 : 0;
-            __syncwarp();
-            if (lane < nd) dvals[rank] = K::to_float(skeys[p]);
-        }
-        __syncthreads();
-    }
+    count_distinct<KeyT, THREADS>(skeys, m, ps);
+    block_prefix_sums<KeyT, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
+    const int nd = ps.misc[0];
+    if (nd <= 16) collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
 
     // ---------------------------------------------------------------- 4./5. Lloyd iterations, error
-    if (warp == 0) {
-        // lane -> (width index bi, centroid index j)
-        int bi = 0, off = 0;
-        while (bi < a.nb && lane >= off + (1 << (a.bmin + bi))) { off += 1 << (a.bmin + bi); ++bi; }
-        const bool in_set = lane < a.sumk;
-        const int width = a.bmin + bi;
-        const int k = 1 << width;
-        const int j = lane - off;
-        const bool wanted = in_set && (!a.row_bits || a.row_bits[row] == width);
-        const bool degenerate = wanted && (nd <= k);      // every value gets its own centroid
-        const bool normal = wanted && !degenerate;
-        float c = 0.0f;
-        if (degenerate) c = dvals[min(j, nd - 1)];
-        if (normal) c = K::to_float(skeys[(int)(((long long)(2 * j + 1) * m) / (2 * k))]);
-
-        int Bprev = -1;
-        float tf = __int_as_float(0x7f800000);            // +inf: no boundary above the last centroid
-        double err_j = 0.0;
-        for (int it = 0;; ++it) {
-            const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
-            int B = m;
-            if (wanted && j < k - 1) {
-                tf = __double2float_rd(0.5 * ((double)c + (double)c_up));
-                if (tf == 0.0f) tf = 0.0f;
-                if (normal) {
-                    const KeyT kt = K::floor_key(tf);
-                    int lo = 0, hi = m;
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        if (skeys[mid] <= kt) lo = mid + 1; else hi = mid;
-                    }
-                    B = lo;
-                }
-            }
-            const bool same = __all_sync(0xffffffffu, B == Bprev);
-            const bool final = (it >= a.iters) || same;
-            Bprev = B;
-            D3 P = {0.0, 0.0, 0.0};
-            if (normal) {
-                const int blk = B >> a.blk_shift;
-                P.a = PB0[blk]; P.b = PB1[blk]; P.c = PB2[blk];
-                for (int u = blk << a.blk_shift; u < B; ++u) {
-                    const double g = (double)sg[u];
-                    const double x = (double)K::to_float(skeys[u]);
-                    const double gx = g * x;
-                    P.a += g;
-                    P.b += gx;
-                    P.c = fma(gx, x, P.c);
-                }
-            }
-            D3 Q = shfl_up3(P, 1);
-            if (j == 0) { Q.a = 0.0; Q.b = 0.0; Q.c = 0.0; }
-            const double S0 = P.a - Q.a, S1 = P.b - Q.b, S2 = P.c - Q.c;
-            if (final) {
-                if (normal) {
-                    const double cd = (double)c;
-                    err_j = fmax(fma(cd, fma(cd, S0, -2.0 * S1), S2), 0.0);
-                }
-                break;
-            }
-            if (normal && S0 > 0.0) c = (float)(S1 / S0);
-        }
-        errs[lane] = err_j;
-        tfs[lane] = (wanted && j < k - 1) ? tf : __int_as_float(0x7f800000);
-        __syncwarp();
-        if (wanted) {
-            if (a.centroids) a.centroids[row * a.sumk + lane] = c;
-            if (j == 0 && a.err) {
-                double e = 0.0;
-                for (int u = 0; u < k; ++u) e += errs[lane + u];
-                if (a.row_bits) a.err[row] = (float)e; else a.err[row * a.nb + bi] = (float)e;
-            }
-        }
-    }
+    if (warp == 0) lloyd_warp<KeyT>(skeys, sg, PB, nd, a, row, ps);
     if (!a.codes) return;
     __syncthreads();
-
-    // ---------------------------------------------------------------- optional: labels in column order
-    {
-        int only = -1;
-        if (a.row_bits) only = (int)a.row_bits[row] - a.bmin;
-        for (int e = tid; e < m; e += THREADS) {
-            float x = __half2float(__ushort_as_half(Wr[e]));
-            if (a.rscale) x = __fmul_rn(x, a.rscale[e]);
-            int off = 0;
-            for (int bi = 0; bi < a.nb; ++bi) {
-                const int k = 1 << (a.bmin + bi);
-                if (only < 0 || only == bi) {
-                    int code = 0;
-                    for (int u = 0; u < k - 1; ++u) code += (tfs[off + u] < x) ? 1 : 0;
-                    if (only < 0) a.codes[((int64_t)bi * a.rows + row) * m + e] = (uint8_t)code;
-                    else a.codes[row * (int64_t)m + e] = (uint8_t)code;
-                }
-                off += k;
-            }
-        }
-    }
+    write_codes<THREADS>(a, row, ps);
 }
 
 struct Variant {
@@ -489,6 +260,10 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     a.codes = codes;
     a.err = err;
     a.status = ws.status;
+    if (!scaled) {
+        const int rc16 = skim_launch_cluster16(ctx, a, rows);
+        if (rc16 <= 0) return rc16;     // launched (or failed); 1 means: not applicable here
+    }
     SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     v->kernel<<<(unsigned)rows, v->threads, smem, ctx->stream>>>(a);
     SKIM_CUDA_OK(cudaGetLastError());
