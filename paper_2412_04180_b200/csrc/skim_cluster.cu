@@ -25,7 +25,7 @@ template <> struct Passes<uint16_t> { static constexpr int N = 2; };
 
 // Shared-memory layout, computed identically on host and device.
 struct SmemLayout {
-    size_t keys, gs, uni, dbase, phase, total;
+    size_t keys, gs, uni, gi, dbase, phase, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nwarps, int blk_shift)
@@ -39,6 +39,7 @@ __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nw
     size_t nblk = ((size_t)cap >> blk_shift) + 2;
     size_t prefix = 3 * nblk * 8;
     L.uni = take(counters > prefix ? counters : prefix);
+    L.gi = take((size_t)sk_entries(cap) * key_bytes);
     L.dbase = take(RADIX * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.total = off;
@@ -59,6 +60,7 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + L.uni);
     double *PB = reinterpret_cast<double *>(smem + L.uni);
     uint32_t *dbase = reinterpret_cast<uint32_t *>(smem + L.dbase);
+    KeyT *GI = reinterpret_cast<KeyT *>(smem + L.gi);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
 
     const int tid = threadIdx.x;
@@ -174,12 +176,13 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     if (tid == 0) { ps.misc[0] = 0; ps.misc[1] = 0; }
     __syncthreads();
     count_distinct<KeyT, THREADS>(skeys, m, ps);
+    build_group_index<KeyT, THREADS>(skeys, m, GI);
     block_prefix_sums<KeyT, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
     const int nd = ps.misc[0];
     if (nd <= 16) collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
 
     // ---------------------------------------------------------------- 4./5. Lloyd iterations, error
-    if (warp == 0) lloyd_warp<KeyT>(skeys, sg, PB, nd, a, row, ps);
+    if (warp == 0) lloyd_warp<KeyT>(skeys, sg, PB, GI, nd, a, row, ps);
     if (!a.codes) return;
     __syncthreads();
     write_codes<THREADS>(a, row, ps);

@@ -13,7 +13,7 @@
 //   pass 1  high 6 key bits, stable: lanes holding the same digit are found with 6 ballots.
 //   gather  importance is brought into sorted order through the column index; keys and sorted
 //           importance take over the sort buffers, the block prefix sums the rest.
-//   then    prefix sums, Lloyd iterations, error: skim_cluster_phases.cuh.
+//   then    group index, prefix sums, Lloyd iterations, error: skim_cluster_phases.cuh.
 //
 // Shared memory per 11 008-column row is about 103 KB and the kernel is held to 64 registers, so two
 // rows are resident per SM: one row's latency-bound Lloyd iterations overlap the other's sort.
@@ -28,7 +28,7 @@ constexpr int D1_BITS = 6, D1 = 1 << D1_BITS;
 constexpr int MBAR_SPIN_LIMIT = 1 << 22;
 
 struct Layout16 {
-    size_t buf, graw, uni, dbase1, phase, mbar, total;
+    size_t buf, graw, uni, gi, dbase1, phase, mbar, total;
 };
 
 // buf:  CAP words: packed items during the sort, sorted importance (fp32) afterwards
@@ -46,6 +46,7 @@ __host__ __device__ inline Layout16 layout16(int cap, int nwarps, int blk_shift)
     const size_t pb_in_graw = (size_t)cap * 2;
     const size_t pb_over = pb > pb_in_graw ? pb - pb_in_graw : 0;
     L.uni = take(counters > pb_over ? counters : pb_over);
+    L.gi = take((size_t)sk_entries(cap) * 2);
     L.dbase1 = take(D1 * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.mbar = take(16);
@@ -109,6 +110,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_cluste
     uint32_t *C0 = reinterpret_cast<uint32_t *>(smem + L.uni);
     uint32_t *cnt1 = C0 + D0;
     uint32_t *dbase1 = reinterpret_cast<uint32_t *>(smem + L.dbase1);
+    uint16_t *GI = reinterpret_cast<uint16_t *>(smem + L.gi);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
     uint64_t *mbar = reinterpret_cast<uint64_t *>(smem + L.mbar);
     uint32_t *scratch = reinterpret_cast<uint32_t *>(ps.wtot);
@@ -275,10 +277,11 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_cluste
 
     // ---------------------------------------------------------------- prefix sums, Lloyd, error
     count_distinct<uint16_t, THREADS>(skeys, m, ps);
+    build_group_index<uint16_t, THREADS>(skeys, m, GI);
     block_prefix_sums<uint16_t, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
     const int nd = ps.misc[0];
     if (nd <= 16) collect_distinct<uint16_t, THREADS>(skeys, m, nd, ps);
-    if (warp == 0) lloyd_warp<uint16_t>(skeys, sg, PB, nd, a, row, ps);
+    if (warp == 0) lloyd_warp<uint16_t>(skeys, sg, PB, GI, nd, a, row, ps);
     if (!a.codes) return;
     __syncthreads();
     write_codes<THREADS>(a, row, ps);

@@ -101,24 +101,105 @@ struct PhaseSmem {
     int misc[4];   // [0] distinct count, [1] slot counter
 };
 
-// Adds the first n (0..8) elements of an aligned 8-element group to P, in index order.
-template <typename KeyT>
-__device__ __forceinline__ void add_group8(const KeyT *k8, const float *g8, int n, bool want_c, D3 &P)
-{
-    const float4 ga = *reinterpret_cast<const float4 *>(g8), gb = *reinterpret_cast<const float4 *>(g8 + 4);
-    const float gs[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-    float xs[8];
-    KeyOps<KeyT>::load8(k8, xs);
+// An aligned group of 8 sorted elements (keys and importance) held in registers.
+template <typename KeyT> struct Group8;
+
+template <> struct Group8<uint16_t> {
+    uint4 kv;
+    float4 ga, gb;
+    __device__ __forceinline__ void load(const uint16_t *k8, const float *g8)
+    {
+        kv = *reinterpret_cast<const uint4 *>(k8);
+        ga = *reinterpret_cast<const float4 *>(g8);
+        gb = *reinterpret_cast<const float4 *>(g8 + 4);
+    }
+    // Number of keys <= kt.  A word holds two ascending keys (low half first): "high half <= kt"
+    // is one 32-bit compare against (kt << 16 | 0xffff), "low half <= kt" one compare of the word
+    // shifted left by 16.
+    __device__ __forceinline__ int count_le(uint16_t kt) const
+    {
+        const uint32_t khi = ((uint32_t)kt << 16) | 0xffffu, klo = (uint32_t)kt << 16;
+        const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+        int c = 0;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        if (u < n) {
-            const double g = (double)gs[u], x = (double)xs[u];
-            const double gx = g * x;
-            P.a += g;
-            P.b += gx;
-            if (want_c) P.c = fma(gx, x, P.c);
+        for (int q = 0; q < 4; ++q) c += (w[q] <= khi ? 1 : 0) + ((w[q] << 16) <= klo ? 1 : 0);
+        return c;
+    }
+    __device__ __forceinline__ void values(float *x) const
+    {
+        const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            x[2 * u] = KeyOps<uint16_t>::to_float((uint16_t)(w[u] & 0xffffu));
+            x[2 * u + 1] = KeyOps<uint16_t>::to_float((uint16_t)(w[u] >> 16));
         }
     }
+};
+
+template <> struct Group8<uint32_t> {
+    uint4 ka, kb;
+    float4 ga, gb;
+    __device__ __forceinline__ void load(const uint32_t *k8, const float *g8)
+    {
+        ka = *reinterpret_cast<const uint4 *>(k8);
+        kb = *reinterpret_cast<const uint4 *>(k8 + 4);
+        ga = *reinterpret_cast<const float4 *>(g8);
+        gb = *reinterpret_cast<const float4 *>(g8 + 4);
+    }
+    __device__ __forceinline__ int count_le(uint32_t kt) const
+    {
+        return (ka.x <= kt ? 1 : 0) + (ka.y <= kt ? 1 : 0) + (ka.z <= kt ? 1 : 0) + (ka.w <= kt ? 1 : 0) +
+               (kb.x <= kt ? 1 : 0) + (kb.y <= kt ? 1 : 0) + (kb.z <= kt ? 1 : 0) + (kb.w <= kt ? 1 : 0);
+    }
+    __device__ __forceinline__ void values(float *x) const
+    {
+        using K = KeyOps<uint32_t>;
+        x[0] = K::to_float(ka.x); x[1] = K::to_float(ka.y); x[2] = K::to_float(ka.z); x[3] = K::to_float(ka.w);
+        x[4] = K::to_float(kb.x); x[5] = K::to_float(kb.y); x[6] = K::to_float(kb.z); x[7] = K::to_float(kb.w);
+    }
+};
+
+// Adds the first n (0..8) elements of a group to P.  The eight terms are summed pairwise (a fixed
+// order, short dependency chain) and the group total is added to P.  Elements past n are masked
+// before any arithmetic touches them.
+template <typename KeyT, bool WANT_C>
+__device__ __forceinline__ void add_group(const Group8<KeyT> &grp, int n, D3 &P)
+{
+    const float gs[8] = {grp.ga.x, grp.ga.y, grp.ga.z, grp.ga.w, grp.gb.x, grp.gb.y, grp.gb.z, grp.gb.w};
+    float xs[8];
+    grp.values(xs);
+    double t0[8], t1[8], t2[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const bool in = u < n;
+        const double g = (double)(in ? gs[u] : 0.0f), x = (double)(in ? xs[u] : 0.0f);
+        t0[u] = g;
+        t1[u] = g * x;
+        if (WANT_C) t2[u] = t1[u] * x;
+    }
+    P.a += ((t0[0] + t0[1]) + (t0[2] + t0[3])) + ((t0[4] + t0[5]) + (t0[6] + t0[7]));
+    P.b += ((t1[0] + t1[1]) + (t1[2] + t1[3])) + ((t1[4] + t1[5]) + (t1[6] + t1[7]));
+    if (WANT_C) P.c += ((t2[0] + t2[1]) + (t2[2] + t2[3])) + ((t2[4] + t2[5]) + (t2[6] + t2[7]));
+}
+
+template <typename KeyT, bool WANT_C>
+__device__ __forceinline__ void add_group8(const KeyT *k8, const float *g8, int n, D3 &P)
+{
+    Group8<KeyT> grp;
+    grp.load(k8, g8);
+    add_group<KeyT, WANT_C>(grp, n, P);
+}
+
+// Group index: GI[q] = first key of the q-th group of 8 sorted elements, padded with the largest
+// key to sk_entries(m) entries.  The boundary search of the Lloyd iteration runs over this 8x
+// smaller array first.
+__host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
+
+template <typename KeyT, int THREADS>
+__device__ __forceinline__ void build_group_index(const KeyT *skeys, int m, KeyT *GI)
+{
+    const int ngrp = (m + 7) >> 3, n = sk_entries(m);
+    for (int q = threadIdx.x; q < n; q += THREADS) GI[q] = q < ngrp ? skeys[q << 3] : KeyOps<KeyT>::PAD;
 }
 
 // Number of distinct keys among skeys[0, m) -> ps.misc[0].  Call with all threads; needs a
@@ -155,7 +236,7 @@ __device__ __forceinline__ void block_prefix_sums(const KeyT *skeys, const float
         if (b < b1) {
             const int lo = b << blk_shift;
             const int cnt = min(m - lo, BLK);
-            for (int c = 0; c < BLK; c += 8) add_group8<KeyT>(skeys + lo + c, sg + lo + c, min(max(cnt - c, 0), 8), true, v);
+            for (int c = 0; c < BLK; c += 8) add_group8<KeyT, true>(skeys + lo + c, sg + lo + c, min(max(cnt - c, 0), 8), v);
         }
         D3 inc = v;
 #pragma unroll
@@ -213,52 +294,91 @@ __device__ __forceinline__ void collect_distinct(const KeyT *skeys, int m, int n
     __syncthreads();
 }
 
-// Number of keys <= kt among the sorted skeys[0, m), searched outward from `guess` (the answer of
-// the previous iteration; -1: plain binary search).
-template <typename KeyT>
-__device__ __forceinline__ int upper_bound_near(const KeyT *skeys, int m, KeyT kt, int guess)
+// A window of 16 ascending keys of the group index around the previous boundary position (at
+// least 4 entries, i.e. 32 elements, on either side), held in registers across one Lloyd
+// iteration: the next search needs no shared-memory round trip unless the boundary left it.
+template <typename KeyT> struct KeyWindow;
+
+template <> struct KeyWindow<uint16_t> {
+    static constexpr int N = 16;
+    uint4 v[2];
+    int ws;
+    __device__ __forceinline__ void load(const uint16_t *skeys, int m, int guess)
+    {
+        const int top = ((m + 7) & ~7) - N;
+        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, top));
+        const uint4 *p = reinterpret_cast<const uint4 *>(skeys + ws);
+        v[0] = p[0]; v[1] = p[1];
+    }
+    // number of window keys <= kt.  A word holds two ascending keys (low half first), so
+    // "high half <= kt" is one 32-bit compare against (kt << 16 | 0xffff) and "low half <= kt"
+    // one compare of the word shifted left by 16.
+    __device__ __forceinline__ int count_le(uint16_t kt) const
+    {
+        const uint32_t khi = ((uint32_t)kt << 16) | 0xffffu, klo = (uint32_t)kt << 16;
+        const uint32_t w[8] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w};
+        int c = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) c += (w[q] <= khi ? 1 : 0) + ((w[q] << 16) <= klo ? 1 : 0);
+        return c;
+    }
+};
+
+template <> struct KeyWindow<uint32_t> {
+    static constexpr int N = 16;
+    uint4 v[4];
+    int ws;
+    __device__ __forceinline__ void load(const uint32_t *skeys, int m, int guess)
+    {
+        const int top = ((m + 7) & ~7) - N;
+        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, top));
+        const uint4 *p = reinterpret_cast<const uint4 *>(skeys + ws);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = p[q];
+    }
+    __device__ __forceinline__ int count_le(uint32_t kt) const
+    {
+        int c = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            c += (v[q].x <= kt ? 1 : 0) + (v[q].y <= kt ? 1 : 0) + (v[q].z <= kt ? 1 : 0) + (v[q].w <= kt ? 1 : 0);
+        return c;
+    }
+};
+
+// s1 / s0 for s0 > 0: binary32 reciprocal seed and two binary64 Newton corrections (relative
+// error about 2^-60, i.e. the correctly rounded quotient up to the last bit or so); operands far
+// outside the binary32 range take the plain division.
+__device__ __forceinline__ double quotient(double s1, double s0)
 {
-    int lo = 0, hi = m;
-    if (guess >= 0) {
-        const bool at = guess < m && skeys[guess] <= kt;
-        const bool below = guess > 0 && skeys[guess - 1] > kt;
-        if (at) {
-            lo = guess + 1;
-            for (int step = 1;; step <<= 1) {
-                const int idx = lo + step - 1;
-                if (idx >= m) { hi = m; break; }
-                if (skeys[idx] <= kt) lo = idx + 1; else { hi = idx; break; }
-            }
-        } else if (below) {
-            hi = guess - 1;
-            for (int step = 1;; step <<= 1) {
-                const int idx = hi - step;
-                if (idx < 0) { lo = 0; break; }
-                if (skeys[idx] > kt) hi = idx; else { lo = idx + 1; break; }
-            }
-        } else {
-            return guess;
-        }
-    }
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (skeys[mid] <= kt) lo = mid + 1; else hi = mid;
-    }
-    return lo;
+    const float s0f = (float)s0;
+    if (!(s0f > 1e-30f && s0f < 1e30f) || !(fabs(s1) < 1e30)) return s1 / s0;
+    const float rf = __frcp_rn(s0f);
+    const double rd = (double)rf;
+    double q = (double)((float)s1 * rf);
+    q = fma(fma(-q, s0, s1), rd, q);
+    q = fma(fma(-q, s0, s1), rd, q);
+    return q;
 }
 
 // Lloyd iterations and the error table entry, run by ONE warp (all 32 lanes must call).
 // Lane L owns centroid L of the row's concatenated centroid record and the boundary above it.
-// On return ps.tfs[L] holds that boundary (largest binary32 value still assigned to centroid L).
+// Per iteration a lane: forms the exact midpoint; counts the group-index entries below it in a
+// register window prefetched around the previous position (falling back to a binary search of the
+// group index when the boundary left the window); loads that one group of 8 keys + importance,
+// which gives both the exact boundary position and the ragged part of the prefix sum.
+// On return ps.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
 template <typename KeyT>
-__device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, const double *PB, int nd,
+__device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, const double *PB, const KeyT *GI, int nd,
                                            const ClusterArgs &a, int64_t row, PhaseSmem &ps)
 {
     using K = KeyOps<KeyT>;
+    using Win = KeyWindow<KeyT>;
     const int lane = threadIdx.x & 31;
     const int m = a.m;
     const int BLK = 1 << a.blk_shift;
     const int nblk = (m + BLK - 1) >> a.blk_shift;
+    const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
     const double *PB0 = PB, *PB1 = PB + (nblk + 1), *PB2 = PB + 2 * (nblk + 1);
     int bi = 0, off = 0;
     while (bi < a.nb && lane >= off + (1 << (a.bmin + bi))) { off += 1 << (a.bmin + bi); ++bi; }
@@ -270,6 +390,7 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
     const bool degenerate = wanted && (nd <= k);      // every value gets its own centroid
     const bool normal = wanted && !degenerate;
     const bool has_boundary = wanted && j < k - 1;
+    const bool searches = normal && j < k - 1;
     float c = 0.0f;
     if (degenerate) c = ps.dvals[min(j, nd - 1)];
     if (normal) c = K::to_float(skeys[(int)(((long long)(2 * j + 1) * m) / (2 * k))]);
@@ -277,28 +398,65 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
     int Bprev = -1;
     float tf = __int_as_float(0x7f800000);            // +inf: no boundary above the last centroid
     double err_j = 0.0;
+    Win win;
+    win.ws = 0;
+    bool have_win = false;
     for (int it = 0;; ++it) {
         const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
         int B = m;
+        Group8<KeyT> grp;
+        int gs = 0, cntk = 0;                         // group start and keys of the group <= boundary
         if (has_boundary) {
             // exact midpoint of two binary32 centroids, rounded down to binary32: x <= midpoint
             // holds for a binary32 x exactly when x <= tf
             tf = __double2float_rd(0.5 * ((double)c + (double)c_up));
             if (tf == 0.0f) tf = 0.0f;
-            if (normal) B = upper_bound_near<KeyT>(skeys, m, K::floor_key(tf), Bprev);
+        }
+        if (searches) {
+            const KeyT kt = K::floor_key(tf);
+            int nle = -1;                              // group-index entries <= kt
+            if (have_win) {
+                const int cnt = win.count_le(kt);
+                if ((cnt > 0 || win.ws == 0) && cnt < Win::N) nle = win.ws + cnt;
+            }
+            if (nle < 0) {
+                int lo = 0, hi = ngi;
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (GI[mid] <= kt) lo = mid + 1; else hi = mid;
+                }
+                nle = lo;
+            }
+            gs = max(nle - 1, 0) << 3;
+            grp.load(skeys + gs, sg + gs);
+            cntk = grp.count_le(kt);
+            B = min(gs + cntk, m);
         }
         const bool same = __all_sync(0xffffffffu, B == Bprev);
         const bool final = (it >= a.iters) || same;
         Bprev = B;
         D3 P = {0.0, 0.0, 0.0};
         if (normal) {
-            const int blk = B >> a.blk_shift;
+            // the last centroid of a width has no boundary above it: its prefix is the row total
+            const int blk = searches ? (B >> a.blk_shift) : nblk;
             const int lo = blk << a.blk_shift;
             P.a = PB0[blk];
             P.b = PB1[blk];
             if (final) P.c = PB2[blk];
-            const int cnt = B - lo;
-            for (int q = 0; q < cnt; q += 8) add_group8<KeyT>(skeys + lo + q, sg + lo + q, min(cnt - q, 8), final, P);
+            if (searches) {
+                // elements [lo, B): whole groups before the loaded one (blocks longer than 8 only), then
+                // the first cntk elements of the loaded group
+                const int part = lo <= gs ? cntk : 0;
+                if (final) {
+                    for (int q = lo; q < gs; q += 8) add_group8<KeyT, true>(skeys + q, sg + q, 8, P);
+                    add_group<KeyT, true>(grp, part, P);
+                } else {
+                    for (int q = lo; q < gs; q += 8) add_group8<KeyT, false>(skeys + q, sg + q, 8, P);
+                    add_group<KeyT, false>(grp, part, P);
+                    win.load(GI, ngi, max(gs >> 3, 0) + 1);   // for the next iteration
+                    have_win = true;
+                }
+            }
         }
         D3 Q;
         Q.a = __shfl_up_sync(0xffffffffu, P.a, 1);
@@ -313,7 +471,7 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
             }
             break;
         }
-        if (normal && S0 > 0.0) c = (float)(S1 / S0);
+        if (normal && S0 > 0.0) c = (float)quotient(S1, S0);
     }
     ps.errs[lane] = err_j;
     ps.tfs[lane] = has_boundary ? tf : __int_as_float(0x7f800000);
