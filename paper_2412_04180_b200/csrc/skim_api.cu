@@ -147,7 +147,7 @@ static int cluster_common(skim_ctx *ctx, const uint16_t *W, const float *importa
     rc = check_matrix(ctx, rows, cols, ld);
     if (rc) return rc;
     if (iters < 0) return SKIM_ERR_SHAPE;
-    rc = check_workspace(ctx, 0, cols);
+    rc = check_workspace(ctx, rows, cols);
     if (rc) return rc;
     if (ctx->scaled && ctx->scale_cols != cols) return SKIM_ERR_SCALE;
     DeviceGuard guard(ctx->device);

@@ -1,7 +1,15 @@
-// Generic row-clustering kernel: weighted 1-D K-means of one matrix row at every candidate width
-// (SKIM Algorithm 3, error pre-recording loop; objective of Section 3.2, diagonal form).
-// Handles every case: scaled rows (32-bit keys of the binary32 product) and rows whose layout rules
-// out the vectorised fp16-key kernel of skim_cluster16.cu.
+// Row clustering: weighted 1-D K-means of every matrix row at every candidate width (SKIM
+// Algorithm 3, error pre-recording loop; objective of Section 3.2, diagonal form), in two kernels
+// per chunk of rows: a sort kernel (one block per row) that leaves the sorted row, its group index
+// and its block prefix sums in a row record in global memory, and the Lloyd kernel (skim_lloyd.cu,
+// one warp per row, thousands of rows in flight) that iterates on the records.  The split exists
+// because the Lloyd iteration is a long chain of dependent small steps: inside the sort block it ran
+// on one warp while two rows filled an SM's shared memory; from global memory (the hot lines stay in
+// L1) every SM keeps 32 rows in flight.
+//
+// This file: the generic sort kernel, which handles every case -- scaled rows (32-bit keys of the
+// binary32 product) and rows whose layout rules out the vectorised fp16-key kernel of
+// skim_cluster16.cu -- and the host-side launcher of the whole clustering.
 //
 // One thread block owns one row.
 //   1. load   the row's (value, importance) pairs into registers; the value is turned into an
@@ -9,7 +17,7 @@
 //   2. sort   block-wide LSD radix sort (8-bit digits, warp-private digit counters, ballot-based
 //             stable ranking), exchanging through one shared-memory buffer.  Afterwards every
 //             1-D cluster is a contiguous interval of the sorted row.
-//   3.-5.     prefix sums, Lloyd iterations and the error: see skim_cluster_phases.cuh.
+//   3.        distinct count, group index, block prefix sums (skim_cluster_phases.cuh), row record.
 #include "skim_cluster_phases.cuh"
 
 namespace {
@@ -47,7 +55,7 @@ __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nw
 }
 
 template <typename KeyT, int THREADS, int ITEMS>
-__global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
+__global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
 {
     using K = KeyOps<KeyT>;
     constexpr int PASSES = Passes<KeyT>::N;
@@ -67,7 +75,7 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const int m = a.m;
-    const int64_t row = blockIdx.x;
+    const int64_t row = a.row0 + blockIdx.x;
     const uint16_t *Wr = a.W + row * a.ld;
     const float *Gr = a.G + row * a.ld;
 
@@ -181,11 +189,8 @@ __global__ void __launch_bounds__(THREADS) skim_cluster_kernel(ClusterArgs a)
     const int nd = ps.misc[0];
     if (nd <= 16) collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
 
-    // ---------------------------------------------------------------- 4./5. Lloyd iterations, error
-    if (warp == 0) lloyd_warp<KeyT>(skeys, sg, PB, GI, nd, a, row, ps);
-    if (!a.codes) return;
-    __syncthreads();
-    write_codes<THREADS>(a, row, ps);
+    // ---------------------------------------------------------------- 4. row record for the Lloyd kernel
+    write_row_record<KeyT, THREADS>(a, skeys, sg, GI, PB, nd, ps.dvals);
 }
 
 struct Variant {
@@ -195,7 +200,7 @@ struct Variant {
     void (*kernel)(ClusterArgs);
 };
 
-#define SKIM_VARIANT(KeyT, T, I) {T * I, T, (int)sizeof(KeyT), skim_cluster_kernel<KeyT, T, I>}
+#define SKIM_VARIANT(KeyT, T, I) {T * I, T, (int)sizeof(KeyT), skim_sort_kernel<KeyT, T, I>}
 
 const Variant kVariants32[] = {
     SKIM_VARIANT(uint32_t, 128, 4),  SKIM_VARIANT(uint32_t, 256, 8),  SKIM_VARIANT(uint32_t, 512, 8),
@@ -240,16 +245,12 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
                         int iters, float *centroids, uint8_t *codes, float *err)
 {
     if (rows == 0) return SKIM_OK;
-    SkimWorkspace ws = skim_carve(ctx->ws, 0, 0);
+    SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
     const bool scaled = ctx->scaled;
-    int blk_shift = 3;
-    size_t smem = 0;
-    const Variant *v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &blk_shift, &smem);
-    if (!v) return SKIM_ERR_SHAPE;
     ClusterArgs a;
     a.W = W;
     a.G = importance;
-    a.rscale = scaled ? skim_carve(ctx->ws, 0, ctx->scale_cols).rscale : nullptr;
+    a.rscale = scaled ? ws.rscale : nullptr;
     a.row_bits = row_bits;
     a.rows = rows;
     a.ld = ld;
@@ -258,18 +259,43 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     a.bmin = bits.b_min;
     a.sumk = bits.sumk;
     a.iters = iters;
-    a.blk_shift = blk_shift;
+    a.blk_shift = 3;
     a.centroids = centroids;
     a.codes = codes;
     a.err = err;
     a.status = ws.status;
-    if (!scaled) {
-        const int rc16 = skim_launch_cluster16(ctx, a, rows);
-        if (rc16 <= 0) return rc16;     // launched (or failed); 1 means: not applicable here
+    a.scratch = ws.cluster_scratch;
+    a.rec_stride = 0;
+    a.row0 = 0;
+
+    // plan: the fp16-key sort kernel when it applies, else the generic one
+    bool fast = !scaled && skim_launch_sort16(ctx, a, 0, false) == SKIM_OK;
+    const Variant *v = nullptr;
+    size_t smem = 0;
+    const int key_bytes = scaled ? 4 : 2;
+    if (!fast) {
+        int blk_shift = 3;
+        v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &blk_shift, &smem);
+        if (!v) return SKIM_ERR_SHAPE;
+        a.blk_shift = blk_shift;
+        a.rec_stride = (long long)row_record(a.m, key_bytes, blk_shift).total;
+        SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
-    SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    v->kernel<<<(unsigned)rows, v->threads, smem, ctx->stream>>>(a);
-    SKIM_CUDA_OK(cudaGetLastError());
-    ctx->launches += 1;
+    if ((size_t)a.rec_stride > skim_cluster_record_bytes(cols)) return SKIM_ERR_WORKSPACE;
+
+    for (int64_t row0 = 0; row0 < rows; row0 += SKIM_CLUSTER_CHUNK_ROWS) {
+        const int64_t n = rows - row0 < SKIM_CLUSTER_CHUNK_ROWS ? rows - row0 : SKIM_CLUSTER_CHUNK_ROWS;
+        a.row0 = row0;
+        if (fast) {
+            const int rc = skim_launch_sort16(ctx, a, n, true);
+            if (rc) return rc < 0 ? rc : SKIM_ERR_SHAPE;
+        } else {
+            v->kernel<<<(unsigned)n, v->threads, smem, ctx->stream>>>(a);
+            SKIM_CUDA_OK(cudaGetLastError());
+            ctx->launches += 1;
+        }
+        const int rc = skim_launch_lloyd(ctx, a, n, key_bytes);
+        if (rc) return rc;
+    }
     return SKIM_OK;
 }

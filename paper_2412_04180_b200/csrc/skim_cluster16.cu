@@ -1,4 +1,4 @@
-// fp16-key row-clustering kernel (SKIM Algorithm 3, error pre-recording loop; objective of
+// fp16-key row-sorting kernel, the first half of the row clustering (SKIM Algorithm 3, error pre-recording loop; objective of
 // Section 3.2, diagonal form) for the common case: no scale vector installed, rows 16-byte aligned.
 //
 // With no scale the clustered value IS the fp16 weight, so a 16-bit order-preserving key is exact
@@ -13,10 +13,12 @@
 //   pass 1  high 6 key bits, stable: lanes holding the same digit are found with 6 ballots.
 //   gather  importance is brought into sorted order through the column index; keys and sorted
 //           importance take over the sort buffers, the block prefix sums the rest.
-//   then    group index, prefix sums, Lloyd iterations, error: skim_cluster_phases.cuh.
+//   then    group index and block prefix sums (skim_cluster_phases.cuh); the sorted row and these
+//           tables are written to the row record in global memory, from which the Lloyd kernel
+//           (skim_lloyd.cu) iterates with one warp per row.
 //
-// Shared memory per 11 008-column row is about 103 KB and the kernel is held to 64 registers, so two
-// rows are resident per SM: one row's latency-bound Lloyd iterations overlap the other's sort.
+// Shared memory per 11 008-column row is about 110 KB and the kernel is held to 64 registers, so two
+// rows are resident per SM.
 #include "skim_cluster_phases.cuh"
 
 namespace {
@@ -94,7 +96,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
 }
 
 template <int THREADS, int VEC>
-__global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_cluster16_kernel(ClusterArgs a)
+__global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16_kernel(ClusterArgs a)
 {
     using K = KeyOps<uint16_t>;
     constexpr int ITEMS = VEC * 8;
@@ -117,7 +119,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_cluste
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = a.m;
-    const int64_t row = blockIdx.x;
+    const int64_t row = a.row0 + blockIdx.x;
     const uint16_t *Wr = a.W + row * a.ld;
     const float *Gr = a.G + row * a.ld;
 
@@ -281,10 +283,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_cluste
     block_prefix_sums<uint16_t, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
     const int nd = ps.misc[0];
     if (nd <= 16) collect_distinct<uint16_t, THREADS>(skeys, m, nd, ps);
-    if (warp == 0) lloyd_warp<uint16_t>(skeys, sg, PB, GI, nd, a, row, ps);
-    if (!a.codes) return;
-    __syncthreads();
-    write_codes<THREADS>(a, row, ps);
+    write_row_record<uint16_t, THREADS>(a, skeys, sg, GI, PB, nd, ps.dvals);
 }
 
 struct Variant16 {
@@ -295,7 +294,7 @@ struct Variant16 {
     int smem_set;
 };
 
-#define SKIM_V16(T, V) {T * V * 8, T, skim_cluster16_kernel<T, V>, -1, 0}
+#define SKIM_V16(T, V) {T * V * 8, T, skim_sort16_kernel<T, V>, -1, 0}
 
 Variant16 kVariants[] = {
     SKIM_V16(128, 1), SKIM_V16(256, 1), SKIM_V16(512, 1), SKIM_V16(512, 2), SKIM_V16(512, 3), SKIM_V16(1024, 2),
@@ -304,7 +303,7 @@ Variant16 kVariants[] = {
 
 }  // namespace
 
-int skim_launch_cluster16(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
+int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool launch)
 {
     const int64_t cols = args.m;
     // 128-bit loads of W rows and the bulk copy of importance rows need 16-byte aligned rows
@@ -315,8 +314,10 @@ int skim_launch_cluster16(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
         for (int s = 3; s <= 5; ++s) {
             const Layout16 L = layout16(v.cap, v.threads / 32, s);
             if (L.total > (size_t)ctx->max_smem_optin) continue;
-            ClusterArgs a = args;
-            a.blk_shift = s;
+            args.blk_shift = s;
+            args.rec_stride = (long long)row_record(args.m, 2, s).total;
+            if (!launch) return SKIM_OK;
+            const ClusterArgs a = args;
             if (v.dev_set != ctx->device || v.smem_set != (int)L.total) {
                 SKIM_CUDA_OK(cudaFuncSetAttribute(v.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
                 v.dev_set = ctx->device;

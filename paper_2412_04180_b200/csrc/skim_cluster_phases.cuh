@@ -77,7 +77,68 @@ struct ClusterArgs {
     uint8_t *codes;
     float *err;
     unsigned long long *status;
+    unsigned char *scratch;   // row records of the current chunk (written by the sort kernel, read by the Lloyd kernel)
+    long long rec_stride;     // bytes between row records
+    int64_t row0;             // first row of the current chunk
 };
+
+// Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are
+// multiples of 16 bytes.
+//   hdr   int nd (number of distinct values) at byte 0; float dvals[16] at byte 64
+//   keys  sorted keys, padded to a multiple of 8 elements with the largest key
+//   g     importance in the same order (0 in the padding)
+//   gi    group index, sk_entries(m) keys
+//   pb    binary64 block prefix sums, three arrays of nblk + 1 entries
+struct RowRecord {
+    size_t keys, g, gi, pb, total;
+    size_t keys_bytes, g_bytes, gi_bytes, pb_bytes;
+};
+
+__host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
+
+__host__ __device__ inline RowRecord row_record(int m, int key_bytes, int blk_shift)
+{
+    RowRecord R;
+    const size_t m8 = ((size_t)m + 7) & ~(size_t)7;
+    const size_t nblk = ((size_t)m + ((size_t)1 << blk_shift) - 1) >> blk_shift;
+    R.keys_bytes = m8 * key_bytes;
+    R.g_bytes = m8 * 4;
+    R.gi_bytes = (size_t)sk_entries(m) * key_bytes;
+    R.pb_bytes = (3 * (nblk + 1) * 8 + 15) & ~(size_t)15;
+    size_t off = 128;
+    R.keys = off; off += (R.keys_bytes + 15) & ~(size_t)15;
+    R.g = off; off += R.g_bytes;
+    R.gi = off; off += R.gi_bytes;
+    R.pb = off; off += R.pb_bytes;
+    R.total = (off + 127) & ~(size_t)127;
+    return R;
+}
+
+// Copies `bytes` (a multiple of 16, both pointers 16-byte aligned) with all threads of the block.
+template <int THREADS>
+__device__ __forceinline__ void copy16(void *dst, const void *src, size_t bytes)
+{
+    uint4 *d = reinterpret_cast<uint4 *>(dst);
+    const uint4 *s = reinterpret_cast<const uint4 *>(src);
+    for (size_t i = threadIdx.x; i < bytes / 16; i += THREADS) d[i] = s[i];
+}
+
+// Writes the row record from the block's shared-memory arrays.  Call with all threads, after
+// block_prefix_sums (and collect_distinct when nd <= 16).
+template <typename KeyT, int THREADS>
+__device__ __forceinline__ void write_row_record(const ClusterArgs &a, const KeyT *skeys, const float *sg, const KeyT *GI,
+                                                 const double *PB, int nd, const float *dvals)
+{
+    const RowRecord R = row_record(a.m, (int)sizeof(KeyT), a.blk_shift);
+    unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
+    if (threadIdx.x == 0) *reinterpret_cast<int *>(rec) = nd;
+    if (threadIdx.x < 16) reinterpret_cast<float *>(rec + 64)[threadIdx.x] = nd <= 16 ? dvals[threadIdx.x] : 0.0f;
+    copy16<THREADS>(rec + R.keys, skeys, R.keys_bytes);
+    copy16<THREADS>(rec + R.g, sg, R.g_bytes);
+    copy16<THREADS>(rec + R.gi, GI, R.gi_bytes);
+    copy16<THREADS>(rec + R.pb, PB, R.pb_bytes);
+}
+
 
 struct D3 {
     double a, b, c;
@@ -193,8 +254,6 @@ __device__ __forceinline__ void add_group8(const KeyT *k8, const float *g8, int 
 // Group index: GI[q] = first key of the q-th group of 8 sorted elements, padded with the largest
 // key to sk_entries(m) entries.  The boundary search of the Lloyd iteration runs over this 8x
 // smaller array first.
-__host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
-
 template <typename KeyT, int THREADS>
 __device__ __forceinline__ void build_group_index(const KeyT *skeys, int m, KeyT *GI)
 {
@@ -487,14 +546,13 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
 }
 
 // Optional labels of the final assignment, in column order (test/diagnostic output).
-template <int THREADS>
-__device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, const PhaseSmem &ps)
+__device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, const PhaseSmem &ps, int start, int stride)
 {
     const int m = a.m;
     const uint16_t *Wr = a.W + row * a.ld;
     int only = -1;
     if (a.row_bits) only = (int)a.row_bits[row] - a.bmin;
-    for (int e = threadIdx.x; e < m; e += THREADS) {
+    for (int e = start; e < m; e += stride) {
         float x = __half2float(__ushort_as_half(Wr[e]));
         if (a.rscale) x = __fmul_rn(x, a.rscale[e]);
         int off = 0;
@@ -513,6 +571,9 @@ __device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, c
 
 }  // namespace skimk
 
-// fp16-key kernel (skim_cluster16.cu).  Returns SKIM_OK after launching, or 1 when the call does
-// not meet its requirements (then the generic kernel must be used).
-int skim_launch_cluster16(skim_ctx *ctx, const skimk::ClusterArgs &args, int64_t rows);
+// fp16-key sort kernel (skim_cluster16.cu).  Fills *blk_shift and *rec_bytes when `launch` is false
+// (planning) and launches over `rows` rows otherwise.  Returns SKIM_OK, or 1 when the call does not
+// meet the kernel's requirements (then the generic sort kernel must be used).
+int skim_launch_sort16(skim_ctx *ctx, skimk::ClusterArgs &args, int64_t rows, bool launch);
+// Lloyd kernel (skim_lloyd.cu): one warp per row record.
+int skim_launch_lloyd(skim_ctx *ctx, const skimk::ClusterArgs &args, int64_t rows, int key_bytes);

@@ -34,10 +34,20 @@ struct SkimWorkspace {
     double *ralpha;              // [cols]     1 / alpha (binary64)
     double *loss_part;           // [SKIM_SCALE_MAX_CTAS]
     double *grad_part;           // [SKIM_SCALE_MAX_CTAS][cols]
+    unsigned char *cluster_scratch;  // [min(rows, SKIM_CLUSTER_CHUNK_ROWS)] row records of the clustering
     size_t bytes;
 };
 
 #define SKIM_SCALE_MAX_CTAS 296
+#define SKIM_CLUSTER_CHUNK_ROWS 8192   // rows clustered per sort-kernel / Lloyd-kernel pair
+
+// Upper bound of one row record of the clustering (4-byte keys, 8-element prefix blocks):
+// 128 header + keys 4 B + importance 4 B + group index 0.5 B + prefix sums 3 B per element, rounded.
+__host__ __device__ static inline size_t skim_cluster_record_bytes(int64_t cols)
+{
+    const size_t m8 = ((size_t)cols + 7) & ~(size_t)7;
+    return ((128 + m8 * 8 + (m8 / 8 + 32) * 4 + 3 * (m8 / 8 + 2) * 8 + 64) + 127) & ~(size_t)127;
+}
 
 static inline size_t skim_align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
@@ -56,6 +66,8 @@ static inline SkimWorkspace skim_carve(void *base, int64_t rows, int64_t cols)
     w.ralpha = (double *)take((size_t)cols * 8);
     w.loss_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * 8);
     w.grad_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * (size_t)cols * 8);
+    w.cluster_scratch = (unsigned char *)take((size_t)(rows < SKIM_CLUSTER_CHUNK_ROWS ? rows : SKIM_CLUSTER_CHUNK_ROWS) *
+                                              skim_cluster_record_bytes(cols));
     w.bytes = off;
     return w;
 }
