@@ -278,7 +278,7 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
         v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &blk_shift, &smem);
         if (!v) return SKIM_ERR_SHAPE;
         a.blk_shift = blk_shift;
-        a.rec_stride = (long long)row_record(a.m, key_bytes, blk_shift).total;
+        a.rec_stride = (long long)row_record(a.m, key_bytes).total;
         SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
     if ((size_t)a.rec_stride > skim_cluster_record_bytes(cols)) return SKIM_ERR_WORKSPACE;

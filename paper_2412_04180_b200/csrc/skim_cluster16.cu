@@ -315,7 +315,7 @@ int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool laun
             const Layout16 L = layout16(v.cap, v.threads / 32, s);
             if (L.total > (size_t)ctx->max_smem_optin) continue;
             args.blk_shift = s;
-            args.rec_stride = (long long)row_record(args.m, 2, s).total;
+            args.rec_stride = (long long)row_record(args.m, 2).total;
             if (!launch) return SKIM_OK;
             const ClusterArgs a = args;
             if (v.dev_set != ctx->device || v.smem_set != (int)L.total) {

@@ -1,7 +1,8 @@
-// Phases of the row-clustering kernels that run after the row has been sorted: distinct-value
-// count, binary64 block prefix sums, the one-warp Lloyd iteration for all widths, the error
-// table entry and the optional labels (SKIM Algorithm 3; objective of Section 3.2, diagonal form).
-// Shared by the generic kernel (skim_cluster.cu) and the fp16-key kernel (skim_cluster16.cu).
+// Device code shared by the row-clustering kernels (SKIM Algorithm 3; objective of Section 3.2,
+// diagonal form): order-preserving keys, the phases the sort kernels run once a row is sorted
+// (distinct-value count, group index, binary64 block prefix sums, the row record), and the one-warp
+// Lloyd iteration with the error table entry and the optional labels that the Lloyd kernel runs on
+// a row record.  Used by skim_cluster.cu, skim_cluster16.cu and skim_lloyd.cu.
 #pragma once
 
 #include "skim_internal.cuh"
@@ -84,32 +85,34 @@ struct ClusterArgs {
 
 // Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are
 // multiples of 16 bytes.
-//   hdr   int nd (number of distinct values) at byte 0; float dvals[16] at byte 64
-//   keys  sorted keys, padded to a multiple of 8 elements with the largest key
-//   g     importance in the same order (0 in the padding)
-//   gi    group index, sk_entries(m) keys
-//   pb    binary64 block prefix sums, three arrays of nblk + 1 entries
+//   hdr     int nd (number of distinct values) at byte 0; double totals[3] (sum g, sum g x,
+//           sum g x^2 over the row) at byte 16; float dvals[16] at byte 64
+//   groups  one record per group of 8 sorted elements: 8 keys, 8 importances, and the binary64
+//           exclusive prefix sums of g and g*x at the group's first element.  Everything a boundary
+//           needs in one Lloyd iteration sits in these 64 (16-bit keys) or 80 (32-bit keys) bytes.
+//           The last group is padded with the largest key and zero importance.
+//   gi      group index: first key of every group, sk_entries(m) keys (padded with the largest key)
+//   p2      binary64 exclusive prefix sums of g*x^2 at every group start (ngrp + 1 entries), read
+//           once, for the error
 struct RowRecord {
-    size_t keys, g, gi, pb, total;
-    size_t keys_bytes, g_bytes, gi_bytes, pb_bytes;
+    size_t groups, gi, p2, total;
+    size_t group_bytes, gi_bytes, p2_bytes;
+    int ngrp;
 };
 
 __host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
 
-__host__ __device__ inline RowRecord row_record(int m, int key_bytes, int blk_shift)
+__host__ __device__ inline RowRecord row_record(int m, int key_bytes)
 {
     RowRecord R;
-    const size_t m8 = ((size_t)m + 7) & ~(size_t)7;
-    const size_t nblk = ((size_t)m + ((size_t)1 << blk_shift) - 1) >> blk_shift;
-    R.keys_bytes = m8 * key_bytes;
-    R.g_bytes = m8 * 4;
+    R.ngrp = (m + 7) >> 3;
+    R.group_bytes = (size_t)8 * key_bytes + 32 + 16;
     R.gi_bytes = (size_t)sk_entries(m) * key_bytes;
-    R.pb_bytes = (3 * (nblk + 1) * 8 + 15) & ~(size_t)15;
+    R.p2_bytes = ((size_t)(R.ngrp + 1) * 8 + 15) & ~(size_t)15;
     size_t off = 128;
-    R.keys = off; off += (R.keys_bytes + 15) & ~(size_t)15;
-    R.g = off; off += R.g_bytes;
+    R.groups = off; off += (size_t)R.ngrp * R.group_bytes;
     R.gi = off; off += R.gi_bytes;
-    R.pb = off; off += R.pb_bytes;
+    R.p2 = off; off += R.p2_bytes;
     R.total = (off + 127) & ~(size_t)127;
     return R;
 }
@@ -122,23 +125,6 @@ __device__ __forceinline__ void copy16(void *dst, const void *src, size_t bytes)
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
     for (size_t i = threadIdx.x; i < bytes / 16; i += THREADS) d[i] = s[i];
 }
-
-// Writes the row record from the block's shared-memory arrays.  Call with all threads, after
-// block_prefix_sums (and collect_distinct when nd <= 16).
-template <typename KeyT, int THREADS>
-__device__ __forceinline__ void write_row_record(const ClusterArgs &a, const KeyT *skeys, const float *sg, const KeyT *GI,
-                                                 const double *PB, int nd, const float *dvals)
-{
-    const RowRecord R = row_record(a.m, (int)sizeof(KeyT), a.blk_shift);
-    unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
-    if (threadIdx.x == 0) *reinterpret_cast<int *>(rec) = nd;
-    if (threadIdx.x < 16) reinterpret_cast<float *>(rec + 64)[threadIdx.x] = nd <= 16 ? dvals[threadIdx.x] : 0.0f;
-    copy16<THREADS>(rec + R.keys, skeys, R.keys_bytes);
-    copy16<THREADS>(rec + R.g, sg, R.g_bytes);
-    copy16<THREADS>(rec + R.gi, GI, R.gi_bytes);
-    copy16<THREADS>(rec + R.pb, PB, R.pb_bytes);
-}
-
 
 struct D3 {
     double a, b, c;
@@ -168,6 +154,14 @@ template <typename KeyT> struct Group8;
 template <> struct Group8<uint16_t> {
     uint4 kv;
     float4 ga, gb;
+    // from a group record in global memory (read-only path); also returns its two prefix sums
+    __device__ __forceinline__ double2 load_record(const unsigned char *gr)
+    {
+        kv = __ldg(reinterpret_cast<const uint4 *>(gr));
+        ga = __ldg(reinterpret_cast<const float4 *>(gr + 16));
+        gb = __ldg(reinterpret_cast<const float4 *>(gr + 32));
+        return __ldg(reinterpret_cast<const double2 *>(gr + 48));
+    }
     __device__ __forceinline__ void load(const uint16_t *k8, const float *g8)
     {
         kv = *reinterpret_cast<const uint4 *>(k8);
@@ -200,6 +194,14 @@ template <> struct Group8<uint16_t> {
 template <> struct Group8<uint32_t> {
     uint4 ka, kb;
     float4 ga, gb;
+    __device__ __forceinline__ double2 load_record(const unsigned char *gr)
+    {
+        ka = __ldg(reinterpret_cast<const uint4 *>(gr));
+        kb = __ldg(reinterpret_cast<const uint4 *>(gr + 16));
+        ga = __ldg(reinterpret_cast<const float4 *>(gr + 32));
+        gb = __ldg(reinterpret_cast<const float4 *>(gr + 48));
+        return __ldg(reinterpret_cast<const double2 *>(gr + 64));
+    }
     __device__ __forceinline__ void load(const uint32_t *k8, const float *g8)
     {
         ka = *reinterpret_cast<const uint4 *>(k8);
@@ -353,6 +355,50 @@ __device__ __forceinline__ void collect_distinct(const KeyT *skeys, int m, int n
     __syncthreads();
 }
 
+// Writes the row record from the block's shared-memory arrays (sorted keys and importance padded
+// to whole groups, group index, block prefix sums).  Call with all threads, after
+// block_prefix_sums (and collect_distinct when nd <= 16).
+template <typename KeyT, int THREADS>
+__device__ __forceinline__ void write_row_record(const ClusterArgs &a, const KeyT *skeys, const float *sg, const KeyT *GI,
+                                                 const double *PB, int nd, const float *dvals)
+{
+    const RowRecord R = row_record(a.m, (int)sizeof(KeyT));
+    unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
+    const int BLK = 1 << a.blk_shift;
+    const int nblk = (a.m + BLK - 1) >> a.blk_shift;
+    const double *PB0 = PB, *PB1 = PB + (nblk + 1), *PB2 = PB + 2 * (nblk + 1);
+    if (threadIdx.x == 0) {
+        *reinterpret_cast<int *>(rec) = nd;
+        double *tot = reinterpret_cast<double *>(rec + 16);
+        tot[0] = PB0[nblk]; tot[1] = PB1[nblk]; tot[2] = PB2[nblk];
+    }
+    if (threadIdx.x < 16) reinterpret_cast<float *>(rec + 64)[threadIdx.x] = nd <= 16 ? dvals[threadIdx.x] : 0.0f;
+    double *p2 = reinterpret_cast<double *>(rec + R.p2);
+    for (int q = threadIdx.x; q <= R.ngrp; q += THREADS) {
+        // prefix sums at the start of group q: the block's entry plus the whole groups before q in it
+        if (q == R.ngrp) { p2[q] = PB2[nblk]; break; }
+        const int e = q << 3;
+        const int blk = e >> a.blk_shift;
+        D3 P = {PB0[blk], PB1[blk], PB2[blk]};
+        for (int u = blk << a.blk_shift; u < e; u += 8) add_group8<KeyT, true>(skeys + u, sg + u, 8, P);
+        p2[q] = P.c;
+        {
+            unsigned char *gr = rec + R.groups + (size_t)q * R.group_bytes;
+            constexpr int KB = 8 * (int)sizeof(KeyT);
+            const uint4 *ks = reinterpret_cast<const uint4 *>(skeys + (q << 3));
+            uint4 *kd = reinterpret_cast<uint4 *>(gr);
+#pragma unroll
+            for (int u = 0; u < KB / 16; ++u) kd[u] = ks[u];
+            const uint4 *gsrc = reinterpret_cast<const uint4 *>(sg + (q << 3));
+            uint4 *gd = reinterpret_cast<uint4 *>(gr + KB);
+            gd[0] = gsrc[0];
+            gd[1] = gsrc[1];
+            *reinterpret_cast<double2 *>(gr + KB + 32) = make_double2(P.a, P.b);
+        }
+    }
+    copy16<THREADS>(rec + R.gi, GI, R.gi_bytes);
+}
+
 // A window of 16 ascending keys of the group index around the previous boundary position (at
 // least 4 entries, i.e. 32 elements, on either side), held in registers across one Lloyd
 // iteration: the next search needs no shared-memory round trip unless the boundary left it.
@@ -367,7 +413,7 @@ template <> struct KeyWindow<uint16_t> {
         const int top = ((m + 7) & ~7) - N;
         ws = max(0, min((((guess + 4) >> 3) << 3) - 8, top));
         const uint4 *p = reinterpret_cast<const uint4 *>(skeys + ws);
-        v[0] = p[0]; v[1] = p[1];
+        v[0] = __ldg(p); v[1] = __ldg(p + 1);
     }
     // number of window keys <= kt.  A word holds two ascending keys (low half first), so
     // "high half <= kt" is one 32-bit compare against (kt << 16 | 0xffff) and "low half <= kt"
@@ -393,7 +439,7 @@ template <> struct KeyWindow<uint32_t> {
         ws = max(0, min((((guess + 4) >> 3) << 3) - 8, top));
         const uint4 *p = reinterpret_cast<const uint4 *>(skeys + ws);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) v[q] = p[q];
+        for (int q = 0; q < 4; ++q) v[q] = __ldg(p + q);
     }
     __device__ __forceinline__ int count_le(uint32_t kt) const
     {
@@ -420,25 +466,27 @@ __device__ __forceinline__ double quotient(double s1, double s0)
     return q;
 }
 
-// Lloyd iterations and the error table entry, run by ONE warp (all 32 lanes must call).
+// Lloyd iterations and the error table entry of one row, run by ONE warp on the row record in
+// global memory (all 32 lanes must call).
 // Lane L owns centroid L of the row's concatenated centroid record and the boundary above it.
 // Per iteration a lane: forms the exact midpoint; counts the group-index entries below it in a
 // register window prefetched around the previous position (falling back to a binary search of the
-// group index when the boundary left the window); loads that one group of 8 keys + importance,
-// which gives both the exact boundary position and the ragged part of the prefix sum.
+// group index when the boundary left the window); loads that one group record, which gives the
+// exact boundary position (keys), the prefix sums at the group start and the few elements between.
 // On return ps.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
 template <typename KeyT>
-__device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, const double *PB, const KeyT *GI, int nd,
-                                           const ClusterArgs &a, int64_t row, PhaseSmem &ps)
+__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, int nd, const ClusterArgs &a, int64_t row, PhaseSmem &ps)
 {
     using K = KeyOps<KeyT>;
     using Win = KeyWindow<KeyT>;
     const int lane = threadIdx.x & 31;
     const int m = a.m;
-    const int BLK = 1 << a.blk_shift;
-    const int nblk = (m + BLK - 1) >> a.blk_shift;
+    const RowRecord R = row_record(m, (int)sizeof(KeyT));
+    const unsigned char *groups = rec + R.groups;
+    const KeyT *GI = reinterpret_cast<const KeyT *>(rec + R.gi);
+    const double *P2 = reinterpret_cast<const double *>(rec + R.p2);
+    const double *tot = reinterpret_cast<const double *>(rec + 16);
     const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
-    const double *PB0 = PB, *PB1 = PB + (nblk + 1), *PB2 = PB + 2 * (nblk + 1);
     int bi = 0, off = 0;
     while (bi < a.nb && lane >= off + (1 << (a.bmin + bi))) { off += 1 << (a.bmin + bi); ++bi; }
     const bool in_set = lane < a.sumk;
@@ -452,7 +500,11 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
     const bool searches = normal && j < k - 1;
     float c = 0.0f;
     if (degenerate) c = ps.dvals[min(j, nd - 1)];
-    if (normal) c = K::to_float(skeys[(int)(((long long)(2 * j + 1) * m) / (2 * k))]);
+    if (normal) {
+        const int idx = (int)(((long long)(2 * j + 1) * m) / (2 * k));
+        c = K::to_float(reinterpret_cast<const KeyT *>(groups + (size_t)(idx >> 3) * R.group_bytes)[idx & 7]);
+    }
+    const double tot0 = normal ? tot[0] : 0.0, tot1 = normal ? tot[1] : 0.0;
 
     int Bprev = -1;
     float tf = __int_as_float(0x7f800000);            // +inf: no boundary above the last centroid
@@ -462,9 +514,9 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
     bool have_win = false;
     for (int it = 0;; ++it) {
         const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
-        int B = m;
+        int B = m, grp_i = 0, cntk = 0;
         Group8<KeyT> grp;
-        int gs = 0, cntk = 0;                         // group start and keys of the group <= boundary
+        double2 gp = make_double2(0.0, 0.0);          // prefix sums at the group start
         if (has_boundary) {
             // exact midpoint of two binary32 centroids, rounded down to binary32: x <= midpoint
             // holds for a binary32 x exactly when x <= tf
@@ -482,39 +534,36 @@ __device__ __forceinline__ void lloyd_warp(const KeyT *skeys, const float *sg, c
                 int lo = 0, hi = ngi;
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
-                    if (GI[mid] <= kt) lo = mid + 1; else hi = mid;
+                    if (__ldg(GI + mid) <= kt) lo = mid + 1; else hi = mid;
                 }
                 nle = lo;
             }
-            gs = max(nle - 1, 0) << 3;
-            grp.load(skeys + gs, sg + gs);
+            grp_i = max(nle - 1, 0);
+            gp = grp.load_record(groups + (size_t)grp_i * R.group_bytes);
             cntk = grp.count_le(kt);
-            B = min(gs + cntk, m);
+            B = min((grp_i << 3) + cntk, m);
         }
         const bool same = __all_sync(0xffffffffu, B == Bprev);
         const bool final = (it >= a.iters) || same;
         Bprev = B;
         D3 P = {0.0, 0.0, 0.0};
         if (normal) {
-            // the last centroid of a width has no boundary above it: its prefix is the row total
-            const int blk = searches ? (B >> a.blk_shift) : nblk;
-            const int lo = blk << a.blk_shift;
-            P.a = PB0[blk];
-            P.b = PB1[blk];
-            if (final) P.c = PB2[blk];
             if (searches) {
-                // elements [lo, B): whole groups before the loaded one (blocks longer than 8 only), then
-                // the first cntk elements of the loaded group
-                const int part = lo <= gs ? cntk : 0;
+                P.a = gp.x;
+                P.b = gp.y;
                 if (final) {
-                    for (int q = lo; q < gs; q += 8) add_group8<KeyT, true>(skeys + q, sg + q, 8, P);
-                    add_group<KeyT, true>(grp, part, P);
+                    P.c = __ldg(P2 + grp_i);
+                    add_group<KeyT, true>(grp, cntk, P);
                 } else {
-                    for (int q = lo; q < gs; q += 8) add_group8<KeyT, false>(skeys + q, sg + q, 8, P);
-                    add_group<KeyT, false>(grp, part, P);
-                    win.load(GI, ngi, max(gs >> 3, 0) + 1);   // for the next iteration
+                    add_group<KeyT, false>(grp, cntk, P);
+                    win.load(GI, ngi, grp_i + 1);       // for the next iteration
                     have_win = true;
                 }
+            } else {
+                // the last centroid of a width has no boundary above it: its prefix is the row total
+                P.a = tot0;
+                P.b = tot1;
+                if (final) P.c = tot[2];
             }
         }
         D3 Q;

@@ -41,12 +41,12 @@ struct SkimWorkspace {
 #define SKIM_SCALE_MAX_CTAS 296
 #define SKIM_CLUSTER_CHUNK_ROWS 8192   // rows clustered per sort-kernel / Lloyd-kernel pair
 
-// Upper bound of one row record of the clustering (4-byte keys, 8-element prefix blocks):
-// 128 header + keys 4 B + importance 4 B + group index 0.5 B + prefix sums 3 B per element, rounded.
+// Upper bound of one row record of the clustering (4-byte keys): 128-byte header, 80 bytes per
+// group of 8 elements, group index 0.5 B and one prefix sum 1 B per element, plus rounding.
 __host__ __device__ static inline size_t skim_cluster_record_bytes(int64_t cols)
 {
     const size_t m8 = ((size_t)cols + 7) & ~(size_t)7;
-    return ((128 + m8 * 8 + (m8 / 8 + 32) * 4 + 3 * (m8 / 8 + 2) * 8 + 64) + 127) & ~(size_t)127;
+    return (12 * m8 + 1024 + 127) & ~(size_t)127;
 }
 
 static inline size_t skim_align256(size_t v) { return (v + 255) & ~(size_t)255; }

@@ -5,9 +5,9 @@
 //
 // An iteration is a chain of dependent small steps (midpoint, search, a few loads, a quotient), so a
 // single row cannot go fast; the kernel gets its throughput from the number of rows in flight: 32 warps
-// per SM, each on its own row.  Per iteration a lane touches a 32-byte window of the group index, one
-// group of 8 keys + 8 importances and two prefix-sum entries; these lines move slowly from one
-// iteration to the next and are served by L1.
+// per SM, each on its own row.  Per iteration a lane touches a 32-byte window of the group index and one
+// 64-byte group record (8 keys, 8 importances, two prefix sums); these move slowly from one iteration to
+// the next and are served by L1 through the read-only path.
 #include "skim_cluster_phases.cuh"
 
 namespace {
@@ -25,14 +25,11 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
     if (local >= rows_in_chunk) return;
     PhaseSmem &ps = ps_all[warp];
     const int64_t row = a.row0 + local;
-    const RowRecord R = row_record(a.m, (int)sizeof(KeyT), a.blk_shift);
     const unsigned char *rec = a.scratch + (size_t)local * (size_t)a.rec_stride;
     const int nd = *reinterpret_cast<const int *>(rec);
     if (lane < 16) ps.dvals[lane] = reinterpret_cast<const float *>(rec + 64)[lane];
     __syncwarp();
-    lloyd_warp<KeyT>(reinterpret_cast<const KeyT *>(rec + R.keys), reinterpret_cast<const float *>(rec + R.g),
-                     reinterpret_cast<const double *>(rec + R.pb), reinterpret_cast<const KeyT *>(rec + R.gi), nd, a, row,
-                     ps);
+    lloyd_warp<KeyT>(rec, nd, a, row, ps);
     if (!a.codes) return;
     __syncwarp();
     write_codes(a, row, ps, lane, 32);
