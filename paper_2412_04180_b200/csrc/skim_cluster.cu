@@ -33,7 +33,7 @@ template <> struct Passes<uint16_t> { static constexpr int N = 2; };
 
 // Shared-memory layout, computed identically on host and device.
 struct SmemLayout {
-    size_t keys, gs, uni, gi, dbase, phase, total;
+    size_t keys, gs, uni, dbase, phase, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nwarps, int blk_shift)
@@ -47,7 +47,6 @@ __host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nw
     size_t nblk = ((size_t)cap >> blk_shift) + 2;
     size_t prefix = 3 * nblk * 8;
     L.uni = take(counters > prefix ? counters : prefix);
-    L.gi = take((size_t)sk_entries(cap) * key_bytes);
     L.dbase = take(RADIX * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.total = off;
@@ -68,7 +67,6 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
     uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + L.uni);
     double *PB = reinterpret_cast<double *>(smem + L.uni);
     uint32_t *dbase = reinterpret_cast<uint32_t *>(smem + L.dbase);
-    KeyT *GI = reinterpret_cast<KeyT *>(smem + L.gi);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
 
     const int tid = threadIdx.x;
@@ -184,13 +182,12 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
     if (tid == 0) { ps.misc[0] = 0; ps.misc[1] = 0; }
     __syncthreads();
     count_distinct<KeyT, THREADS>(skeys, m, ps);
-    build_group_index<KeyT, THREADS>(skeys, m, GI);
     block_prefix_sums<KeyT, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
     const int nd = ps.misc[0];
     if (nd <= 16) collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
 
     // ---------------------------------------------------------------- 4. row record for the Lloyd kernel
-    write_row_record<KeyT, THREADS>(a, skeys, sg, GI, PB, nd, ps.dvals);
+    write_row_record<KeyT, THREADS>(a, skeys, sg, PB, nd, ps.dvals);
 }
 
 struct Variant {
@@ -272,13 +269,12 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     bool fast = !scaled && skim_launch_sort16(ctx, a, 0, false) == SKIM_OK;
     const Variant *v = nullptr;
     size_t smem = 0;
-    const int key_bytes = scaled ? 4 : 2;
     if (!fast) {
         int blk_shift = 3;
         v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &blk_shift, &smem);
         if (!v) return SKIM_ERR_SHAPE;
         a.blk_shift = blk_shift;
-        a.rec_stride = (long long)row_record(a.m, key_bytes).total;
+        a.rec_stride = (long long)row_record(a.m).total;
         SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
     if ((size_t)a.rec_stride > skim_cluster_record_bytes(cols)) return SKIM_ERR_WORKSPACE;
@@ -294,7 +290,7 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
             SKIM_CUDA_OK(cudaGetLastError());
             ctx->launches += 1;
         }
-        const int rc = skim_launch_lloyd(ctx, a, n, key_bytes);
+        const int rc = skim_launch_lloyd(ctx, a, n);
         if (rc) return rc;
     }
     return SKIM_OK;

@@ -13,9 +13,9 @@
 //   pass 1  high 6 key bits, stable: lanes holding the same digit are found with 6 ballots.
 //   gather  importance is brought into sorted order through the column index; keys and sorted
 //           importance take over the sort buffers, the block prefix sums the rest.
-//   then    group index and block prefix sums (skim_cluster_phases.cuh); the sorted row and these
-//           tables are written to the row record in global memory, from which the Lloyd kernel
-//           (skim_lloyd.cu) iterates with one warp per row.
+//   then    block prefix sums (skim_cluster_phases.cuh); the sorted row, its group index and the
+//           prefix sums are written to the row record in global memory, from which the Lloyd
+//           kernel (skim_lloyd.cu) iterates with one warp per row.
 //
 // Shared memory per 11 008-column row is about 110 KB and the kernel is held to 64 registers, so two
 // rows are resident per SM.
@@ -30,7 +30,7 @@ constexpr int D1_BITS = 6, D1 = 1 << D1_BITS;
 constexpr int MBAR_SPIN_LIMIT = 1 << 22;
 
 struct Layout16 {
-    size_t buf, graw, uni, gi, dbase1, phase, mbar, total;
+    size_t buf, graw, uni, dbase1, phase, mbar, total;
 };
 
 // buf:  CAP words: packed items during the sort, sorted importance (fp32) afterwards
@@ -48,7 +48,6 @@ __host__ __device__ inline Layout16 layout16(int cap, int nwarps, int blk_shift)
     const size_t pb_in_graw = (size_t)cap * 2;
     const size_t pb_over = pb > pb_in_graw ? pb - pb_in_graw : 0;
     L.uni = take(counters > pb_over ? counters : pb_over);
-    L.gi = take((size_t)sk_entries(cap) * 2);
     L.dbase1 = take(D1 * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.mbar = take(16);
@@ -112,7 +111,6 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     uint32_t *C0 = reinterpret_cast<uint32_t *>(smem + L.uni);
     uint32_t *cnt1 = C0 + D0;
     uint32_t *dbase1 = reinterpret_cast<uint32_t *>(smem + L.dbase1);
-    uint16_t *GI = reinterpret_cast<uint16_t *>(smem + L.gi);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
     uint64_t *mbar = reinterpret_cast<uint64_t *>(smem + L.mbar);
     uint32_t *scratch = reinterpret_cast<uint32_t *>(ps.wtot);
@@ -279,11 +277,10 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
 
     // ---------------------------------------------------------------- prefix sums, Lloyd, error
     count_distinct<uint16_t, THREADS>(skeys, m, ps);
-    build_group_index<uint16_t, THREADS>(skeys, m, GI);
     block_prefix_sums<uint16_t, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
     const int nd = ps.misc[0];
     if (nd <= 16) collect_distinct<uint16_t, THREADS>(skeys, m, nd, ps);
-    write_row_record<uint16_t, THREADS>(a, skeys, sg, GI, PB, nd, ps.dvals);
+    write_row_record<uint16_t, THREADS>(a, skeys, sg, PB, nd, ps.dvals);
 }
 
 struct Variant16 {
@@ -315,7 +312,7 @@ int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool laun
             const Layout16 L = layout16(v.cap, v.threads / 32, s);
             if (L.total > (size_t)ctx->max_smem_optin) continue;
             args.blk_shift = s;
-            args.rec_stride = (long long)row_record(args.m, 2).total;
+            args.rec_stride = (long long)row_record(args.m).total;
             if (!launch) return SKIM_OK;
             const ClusterArgs a = args;
             if (v.dev_set != ctx->device || v.smem_set != (int)L.total) {

@@ -84,33 +84,33 @@ struct ClusterArgs {
 };
 
 // Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are
-// multiples of 16 bytes.
+// multiples of 16 bytes; values are binary32 whatever key type sorted the row.
 //   hdr     int nd (number of distinct values) at byte 0; double totals[3] (sum g, sum g x,
 //           sum g x^2 over the row) at byte 16; float dvals[16] at byte 64
-//   groups  one record per group of 8 sorted elements: 8 keys, 8 importances, and the binary64
-//           exclusive prefix sums of g and g*x at the group's first element.  Everything a boundary
-//           needs in one Lloyd iteration sits in these 64 (16-bit keys) or 80 (32-bit keys) bytes.
-//           The last group is padded with the largest key and zero importance.
-//   gi      group index: first key of every group, sk_entries(m) keys (padded with the largest key)
+//   groups  one 80-byte record per group of 8 sorted elements: 8 values, 8 importances, and the
+//           binary64 exclusive prefix sums of g and g*x at the group's first element: everything
+//           a boundary needs in one Lloyd iteration.  The last group is padded with the largest
+//           finite value and zero importance.
+//   gi      group index: first value of every group, sk_entries(m) floats (padded likewise)
 //   p2      binary64 exclusive prefix sums of g*x^2 at every group start (ngrp + 1 entries), read
 //           once, for the error
 struct RowRecord {
     size_t groups, gi, p2, total;
-    size_t group_bytes, gi_bytes, p2_bytes;
+    size_t gi_bytes, p2_bytes;
     int ngrp;
 };
+constexpr int SKIM_GROUP_BYTES = 80;
 
 __host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
 
-__host__ __device__ inline RowRecord row_record(int m, int key_bytes)
+__host__ __device__ inline RowRecord row_record(int m)
 {
     RowRecord R;
     R.ngrp = (m + 7) >> 3;
-    R.group_bytes = (size_t)8 * key_bytes + 32 + 16;
-    R.gi_bytes = (size_t)sk_entries(m) * key_bytes;
+    R.gi_bytes = (size_t)sk_entries(m) * 4;
     R.p2_bytes = ((size_t)(R.ngrp + 1) * 8 + 15) & ~(size_t)15;
     size_t off = 128;
-    R.groups = off; off += (size_t)R.ngrp * R.group_bytes;
+    R.groups = off; off += (size_t)R.ngrp * SKIM_GROUP_BYTES;
     R.gi = off; off += R.gi_bytes;
     R.p2 = off; off += R.p2_bytes;
     R.total = (off + 127) & ~(size_t)127;
@@ -142,10 +142,9 @@ __device__ __forceinline__ D3 shfl_up3(D3 v, int off)
 // Small per-block scratch of the phases below.
 struct PhaseSmem {
     double wtot[32 * 3];
-    double errs[32];
-    float tfs[32];
-    float dvals[32];
-    int misc[4];   // [0] distinct count, [1] slot counter
+    float tfs[32];     // scratch of collect_distinct
+    float dvals[32];   // the row's distinct values when there are at most 16
+    int misc[4];       // [0] distinct count, [1] slot counter
 };
 
 // An aligned group of 8 sorted elements (keys and importance) held in registers.
@@ -154,14 +153,6 @@ template <typename KeyT> struct Group8;
 template <> struct Group8<uint16_t> {
     uint4 kv;
     float4 ga, gb;
-    // from a group record in global memory (read-only path); also returns its two prefix sums
-    __device__ __forceinline__ double2 load_record(const unsigned char *gr)
-    {
-        kv = __ldg(reinterpret_cast<const uint4 *>(gr));
-        ga = __ldg(reinterpret_cast<const float4 *>(gr + 16));
-        gb = __ldg(reinterpret_cast<const float4 *>(gr + 32));
-        return __ldg(reinterpret_cast<const double2 *>(gr + 48));
-    }
     __device__ __forceinline__ void load(const uint16_t *k8, const float *g8)
     {
         kv = *reinterpret_cast<const uint4 *>(k8);
@@ -194,14 +185,6 @@ template <> struct Group8<uint16_t> {
 template <> struct Group8<uint32_t> {
     uint4 ka, kb;
     float4 ga, gb;
-    __device__ __forceinline__ double2 load_record(const unsigned char *gr)
-    {
-        ka = __ldg(reinterpret_cast<const uint4 *>(gr));
-        kb = __ldg(reinterpret_cast<const uint4 *>(gr + 16));
-        ga = __ldg(reinterpret_cast<const float4 *>(gr + 32));
-        gb = __ldg(reinterpret_cast<const float4 *>(gr + 48));
-        return __ldg(reinterpret_cast<const double2 *>(gr + 64));
-    }
     __device__ __forceinline__ void load(const uint32_t *k8, const float *g8)
     {
         ka = *reinterpret_cast<const uint4 *>(k8);
@@ -251,16 +234,6 @@ __device__ __forceinline__ void add_group8(const KeyT *k8, const float *g8, int 
     Group8<KeyT> grp;
     grp.load(k8, g8);
     add_group<KeyT, WANT_C>(grp, n, P);
-}
-
-// Group index: GI[q] = first key of the q-th group of 8 sorted elements, padded with the largest
-// key to sk_entries(m) entries.  The boundary search of the Lloyd iteration runs over this 8x
-// smaller array first.
-template <typename KeyT, int THREADS>
-__device__ __forceinline__ void build_group_index(const KeyT *skeys, int m, KeyT *GI)
-{
-    const int ngrp = (m + 7) >> 3, n = sk_entries(m);
-    for (int q = threadIdx.x; q < n; q += THREADS) GI[q] = q < ngrp ? skeys[q << 3] : KeyOps<KeyT>::PAD;
 }
 
 // Number of distinct keys among skeys[0, m) -> ps.misc[0].  Call with all threads; needs a
@@ -356,17 +329,18 @@ __device__ __forceinline__ void collect_distinct(const KeyT *skeys, int m, int n
 }
 
 // Writes the row record from the block's shared-memory arrays (sorted keys and importance padded
-// to whole groups, group index, block prefix sums).  Call with all threads, after
-// block_prefix_sums (and collect_distinct when nd <= 16).
+// to whole groups, block prefix sums).  Call with all threads, after block_prefix_sums (and
+// collect_distinct when nd <= 16).
 template <typename KeyT, int THREADS>
-__device__ __forceinline__ void write_row_record(const ClusterArgs &a, const KeyT *skeys, const float *sg, const KeyT *GI,
-                                                 const double *PB, int nd, const float *dvals)
+__device__ __forceinline__ void write_row_record(const ClusterArgs &a, const KeyT *skeys, const float *sg, const double *PB,
+                                                 int nd, const float *dvals)
 {
-    const RowRecord R = row_record(a.m, (int)sizeof(KeyT));
+    const RowRecord R = row_record(a.m);
     unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
     const int BLK = 1 << a.blk_shift;
     const int nblk = (a.m + BLK - 1) >> a.blk_shift;
     const double *PB0 = PB, *PB1 = PB + (nblk + 1), *PB2 = PB + 2 * (nblk + 1);
+    const float INF = 3.402823466e38f;   // padding value: the largest finite binary32 (0 * padding stays 0)
     if (threadIdx.x == 0) {
         *reinterpret_cast<int *>(rec) = nd;
         double *tot = reinterpret_cast<double *>(rec + 16);
@@ -374,255 +348,42 @@ __device__ __forceinline__ void write_row_record(const ClusterArgs &a, const Key
     }
     if (threadIdx.x < 16) reinterpret_cast<float *>(rec + 64)[threadIdx.x] = nd <= 16 ? dvals[threadIdx.x] : 0.0f;
     double *p2 = reinterpret_cast<double *>(rec + R.p2);
-    for (int q = threadIdx.x; q <= R.ngrp; q += THREADS) {
+    float *gi = reinterpret_cast<float *>(rec + R.gi);
+    for (int q = threadIdx.x; q < sk_entries(a.m); q += THREADS) {
+        if (q >= R.ngrp) {                      // padding of the group index; totals close the p2 array
+            gi[q] = INF;
+            if (q == R.ngrp) p2[q] = PB2[nblk];
+            continue;
+        }
         // prefix sums at the start of group q: the block's entry plus the whole groups before q in it
-        if (q == R.ngrp) { p2[q] = PB2[nblk]; break; }
         const int e = q << 3;
         const int blk = e >> a.blk_shift;
         D3 P = {PB0[blk], PB1[blk], PB2[blk]};
         for (int u = blk << a.blk_shift; u < e; u += 8) add_group8<KeyT, true>(skeys + u, sg + u, 8, P);
         p2[q] = P.c;
-        {
-            unsigned char *gr = rec + R.groups + (size_t)q * R.group_bytes;
-            constexpr int KB = 8 * (int)sizeof(KeyT);
-            const uint4 *ks = reinterpret_cast<const uint4 *>(skeys + (q << 3));
-            uint4 *kd = reinterpret_cast<uint4 *>(gr);
+        float x[8];
+        KeyOps<KeyT>::load8(skeys + e, x);
 #pragma unroll
-            for (int u = 0; u < KB / 16; ++u) kd[u] = ks[u];
-            const uint4 *gsrc = reinterpret_cast<const uint4 *>(sg + (q << 3));
-            uint4 *gd = reinterpret_cast<uint4 *>(gr + KB);
-            gd[0] = gsrc[0];
-            gd[1] = gsrc[1];
-            *reinterpret_cast<double2 *>(gr + KB + 32) = make_double2(P.a, P.b);
+        for (int u = 0; u < 8; ++u) {
+            if (e + u >= a.m) x[u] = INF;
         }
-    }
-    copy16<THREADS>(rec + R.gi, GI, R.gi_bytes);
-}
-
-// A window of 16 ascending keys of the group index around the previous boundary position (at
-// least 4 entries, i.e. 32 elements, on either side), held in registers across one Lloyd
-// iteration: the next search needs no shared-memory round trip unless the boundary left it.
-template <typename KeyT> struct KeyWindow;
-
-template <> struct KeyWindow<uint16_t> {
-    static constexpr int N = 16;
-    uint4 v[2];
-    int ws;
-    __device__ __forceinline__ void load(const uint16_t *skeys, int m, int guess)
-    {
-        const int top = ((m + 7) & ~7) - N;
-        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, top));
-        const uint4 *p = reinterpret_cast<const uint4 *>(skeys + ws);
-        v[0] = __ldg(p); v[1] = __ldg(p + 1);
-    }
-    // number of window keys <= kt.  A word holds two ascending keys (low half first), so
-    // "high half <= kt" is one 32-bit compare against (kt << 16 | 0xffff) and "low half <= kt"
-    // one compare of the word shifted left by 16.
-    __device__ __forceinline__ int count_le(uint16_t kt) const
-    {
-        const uint32_t khi = ((uint32_t)kt << 16) | 0xffffu, klo = (uint32_t)kt << 16;
-        const uint32_t w[8] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w};
-        int c = 0;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) c += (w[q] <= khi ? 1 : 0) + ((w[q] << 16) <= klo ? 1 : 0);
-        return c;
-    }
-};
-
-template <> struct KeyWindow<uint32_t> {
-    static constexpr int N = 16;
-    uint4 v[4];
-    int ws;
-    __device__ __forceinline__ void load(const uint32_t *skeys, int m, int guess)
-    {
-        const int top = ((m + 7) & ~7) - N;
-        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, top));
-        const uint4 *p = reinterpret_cast<const uint4 *>(skeys + ws);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) v[q] = __ldg(p + q);
-    }
-    __device__ __forceinline__ int count_le(uint32_t kt) const
-    {
-        int c = 0;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            c += (v[q].x <= kt ? 1 : 0) + (v[q].y <= kt ? 1 : 0) + (v[q].z <= kt ? 1 : 0) + (v[q].w <= kt ? 1 : 0);
-        return c;
-    }
-};
-
-// s1 / s0 for s0 > 0: binary32 reciprocal seed and two binary64 Newton corrections (relative
-// error about 2^-60, i.e. the correctly rounded quotient up to the last bit or so); operands far
-// outside the binary32 range take the plain division.
-__device__ __forceinline__ double quotient(double s1, double s0)
-{
-    const float s0f = (float)s0;
-    if (!(s0f > 1e-30f && s0f < 1e30f) || !(fabs(s1) < 1e30)) return s1 / s0;
-    const float rf = __frcp_rn(s0f);
-    const double rd = (double)rf;
-    double q = (double)((float)s1 * rf);
-    q = fma(fma(-q, s0, s1), rd, q);
-    q = fma(fma(-q, s0, s1), rd, q);
-    return q;
-}
-
-// Lloyd iterations and the error table entry of one row, run by ONE warp on the row record in
-// global memory (all 32 lanes must call).
-// Lane L owns centroid L of the row's concatenated centroid record and the boundary above it.
-// Per iteration a lane: forms the exact midpoint; counts the group-index entries below it in a
-// register window prefetched around the previous position (falling back to a binary search of the
-// group index when the boundary left the window); loads that one group record, which gives the
-// exact boundary position (keys), the prefix sums at the group start and the few elements between.
-// On return ps.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
-template <typename KeyT>
-__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, int nd, const ClusterArgs &a, int64_t row, PhaseSmem &ps)
-{
-    using K = KeyOps<KeyT>;
-    using Win = KeyWindow<KeyT>;
-    const int lane = threadIdx.x & 31;
-    const int m = a.m;
-    const RowRecord R = row_record(m, (int)sizeof(KeyT));
-    const unsigned char *groups = rec + R.groups;
-    const KeyT *GI = reinterpret_cast<const KeyT *>(rec + R.gi);
-    const double *P2 = reinterpret_cast<const double *>(rec + R.p2);
-    const double *tot = reinterpret_cast<const double *>(rec + 16);
-    const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
-    int bi = 0, off = 0;
-    while (bi < a.nb && lane >= off + (1 << (a.bmin + bi))) { off += 1 << (a.bmin + bi); ++bi; }
-    const bool in_set = lane < a.sumk;
-    const int width = a.bmin + bi;
-    const int k = 1 << width;
-    const int j = lane - off;
-    const bool wanted = in_set && (!a.row_bits || a.row_bits[row] == width);
-    const bool degenerate = wanted && (nd <= k);      // every value gets its own centroid
-    const bool normal = wanted && !degenerate;
-    const bool has_boundary = wanted && j < k - 1;
-    const bool searches = normal && j < k - 1;
-    float c = 0.0f;
-    if (degenerate) c = ps.dvals[min(j, nd - 1)];
-    if (normal) {
-        const int idx = (int)(((long long)(2 * j + 1) * m) / (2 * k));
-        c = K::to_float(reinterpret_cast<const KeyT *>(groups + (size_t)(idx >> 3) * R.group_bytes)[idx & 7]);
-    }
-    const double tot0 = normal ? tot[0] : 0.0, tot1 = normal ? tot[1] : 0.0;
-
-    int Bprev = -1;
-    float tf = __int_as_float(0x7f800000);            // +inf: no boundary above the last centroid
-    double err_j = 0.0;
-    Win win;
-    win.ws = 0;
-    bool have_win = false;
-    for (int it = 0;; ++it) {
-        const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
-        int B = m, grp_i = 0, cntk = 0;
-        Group8<KeyT> grp;
-        double2 gp = make_double2(0.0, 0.0);          // prefix sums at the group start
-        if (has_boundary) {
-            // exact midpoint of two binary32 centroids, rounded down to binary32: x <= midpoint
-            // holds for a binary32 x exactly when x <= tf
-            tf = __double2float_rd(0.5 * ((double)c + (double)c_up));
-            if (tf == 0.0f) tf = 0.0f;
-        }
-        if (searches) {
-            const KeyT kt = K::floor_key(tf);
-            int nle = -1;                              // group-index entries <= kt
-            if (have_win) {
-                const int cnt = win.count_le(kt);
-                if ((cnt > 0 || win.ws == 0) && cnt < Win::N) nle = win.ws + cnt;
-            }
-            if (nle < 0) {
-                int lo = 0, hi = ngi;
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (__ldg(GI + mid) <= kt) lo = mid + 1; else hi = mid;
-                }
-                nle = lo;
-            }
-            grp_i = max(nle - 1, 0);
-            gp = grp.load_record(groups + (size_t)grp_i * R.group_bytes);
-            cntk = grp.count_le(kt);
-            B = min((grp_i << 3) + cntk, m);
-        }
-        const bool same = __all_sync(0xffffffffu, B == Bprev);
-        const bool final = (it >= a.iters) || same;
-        Bprev = B;
-        D3 P = {0.0, 0.0, 0.0};
-        if (normal) {
-            if (searches) {
-                P.a = gp.x;
-                P.b = gp.y;
-                if (final) {
-                    P.c = __ldg(P2 + grp_i);
-                    add_group<KeyT, true>(grp, cntk, P);
-                } else {
-                    add_group<KeyT, false>(grp, cntk, P);
-                    win.load(GI, ngi, grp_i + 1);       // for the next iteration
-                    have_win = true;
-                }
-            } else {
-                // the last centroid of a width has no boundary above it: its prefix is the row total
-                P.a = tot0;
-                P.b = tot1;
-                if (final) P.c = tot[2];
-            }
-        }
-        D3 Q;
-        Q.a = __shfl_up_sync(0xffffffffu, P.a, 1);
-        Q.b = __shfl_up_sync(0xffffffffu, P.b, 1);
-        Q.c = final ? __shfl_up_sync(0xffffffffu, P.c, 1) : 0.0;
-        if (j == 0) { Q.a = 0.0; Q.b = 0.0; Q.c = 0.0; }
-        const double S0 = P.a - Q.a, S1 = P.b - Q.b;
-        if (final) {
-            if (normal) {
-                const double cd = (double)c, S2 = P.c - Q.c;
-                err_j = fmax(fma(cd, fma(cd, S0, -2.0 * S1), S2), 0.0);
-            }
-            break;
-        }
-        if (normal && S0 > 0.0) c = (float)quotient(S1, S0);
-    }
-    ps.errs[lane] = err_j;
-    ps.tfs[lane] = has_boundary ? tf : __int_as_float(0x7f800000);
-    __syncwarp();
-    if (wanted) {
-        if (a.centroids) a.centroids[row * a.sumk + lane] = c;
-        if (j == 0 && a.err) {
-            double e = 0.0;
-            for (int u = 0; u < k; ++u) e += ps.errs[lane + u];
-            if (a.row_bits) a.err[row] = (float)e; else a.err[row * a.nb + bi] = (float)e;
-        }
-    }
-}
-
-// Optional labels of the final assignment, in column order (test/diagnostic output).
-__device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, const PhaseSmem &ps, int start, int stride)
-{
-    const int m = a.m;
-    const uint16_t *Wr = a.W + row * a.ld;
-    int only = -1;
-    if (a.row_bits) only = (int)a.row_bits[row] - a.bmin;
-    for (int e = start; e < m; e += stride) {
-        float x = __half2float(__ushort_as_half(Wr[e]));
-        if (a.rscale) x = __fmul_rn(x, a.rscale[e]);
-        int off = 0;
-        for (int bi = 0; bi < a.nb; ++bi) {
-            const int k = 1 << (a.bmin + bi);
-            if (only < 0 || only == bi) {
-                int code = 0;
-                for (int u = 0; u < k - 1; ++u) code += (ps.tfs[off + u] < x) ? 1 : 0;
-                if (only < 0) a.codes[((int64_t)bi * a.rows + row) * m + e] = (uint8_t)code;
-                else a.codes[row * (int64_t)m + e] = (uint8_t)code;
-            }
-            off += k;
-        }
+        gi[q] = x[0];
+        unsigned char *gr = rec + R.groups + (size_t)q * SKIM_GROUP_BYTES;
+        float4 *xd = reinterpret_cast<float4 *>(gr);
+        xd[0] = make_float4(x[0], x[1], x[2], x[3]);
+        xd[1] = make_float4(x[4], x[5], x[6], x[7]);
+        const float4 *gsrc = reinterpret_cast<const float4 *>(sg + e);
+        xd[2] = gsrc[0];
+        xd[3] = gsrc[1];
+        *reinterpret_cast<double2 *>(gr + 64) = make_double2(P.a, P.b);
     }
 }
 
 }  // namespace skimk
 
-// fp16-key sort kernel (skim_cluster16.cu).  Fills *blk_shift and *rec_bytes when `launch` is false
-// (planning) and launches over `rows` rows otherwise.  Returns SKIM_OK, or 1 when the call does not
-// meet the kernel's requirements (then the generic sort kernel must be used).
+// fp16-key sort kernel (skim_cluster16.cu).  Fills args.blk_shift and args.rec_stride when `launch`
+// is false (planning) and launches over `rows` rows otherwise.  Returns SKIM_OK, or 1 when the
+// call does not meet the kernel's requirements (then the generic sort kernel must be used).
 int skim_launch_sort16(skim_ctx *ctx, skimk::ClusterArgs &args, int64_t rows, bool launch);
 // Lloyd kernel (skim_lloyd.cu): one warp per row record.
-int skim_launch_lloyd(skim_ctx *ctx, const skimk::ClusterArgs &args, int64_t rows, int key_bytes);
+int skim_launch_lloyd(skim_ctx *ctx, const skimk::ClusterArgs &args, int64_t rows);

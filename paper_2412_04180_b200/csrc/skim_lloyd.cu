@@ -1,13 +1,14 @@
 // Lloyd kernel, the second half of the row clustering (SKIM Algorithm 3, error pre-recording loop;
 // objective of Section 3.2, diagonal form): one warp per row iterates on the row record the sort
-// kernel left in global memory (sorted keys and importance, group index, binary64 block prefix sums)
-// and writes the row's centroids and error table entries.
+// kernel left in global memory (sorted values and importance by groups of 8 with their binary64
+// prefix sums, a group index) and writes the row's centroids and error table entries.
 //
 // An iteration is a chain of dependent small steps (midpoint, search, a few loads, a quotient), so a
-// single row cannot go fast; the kernel gets its throughput from the number of rows in flight: 32 warps
-// per SM, each on its own row.  Per iteration a lane touches a 32-byte window of the group index and one
-// 64-byte group record (8 keys, 8 importances, two prefix sums); these move slowly from one iteration to
-// the next and are served by L1 through the read-only path.
+// single row cannot go fast; the kernel gets its throughput from the number of rows in flight: up to 32
+// warps per SM, each on its own row.  A warp first copies its row's group index (4 bytes per 8
+// elements) into shared memory, so that the boundary search never waits on global memory; per
+// iteration a lane then reads one 80-byte group record through the read-only path, the one global
+// round trip of the iteration.
 #include "skim_cluster_phases.cuh"
 
 namespace {
@@ -15,35 +16,284 @@ namespace {
 using namespace skimk;
 
 constexpr int LLOYD_WARPS = 4;   // rows per block
+constexpr int WIN = 16;          // group-index entries held in registers
 
-template <typename KeyT>
+struct LloydSmem {
+    double errs[32];
+    float tfs[32];
+    float dvals[16];
+};
+
+// One group record in registers.
+struct Group {
+    float4 xa, xb, ga, gb;
+    double2 p;   // prefix sums of g and g*x at the group's first element
+    __device__ __forceinline__ void load(const unsigned char *gr)
+    {
+        const float4 *q = reinterpret_cast<const float4 *>(gr);
+        xa = __ldg(q); xb = __ldg(q + 1); ga = __ldg(q + 2); gb = __ldg(q + 3);
+        p = __ldg(reinterpret_cast<const double2 *>(gr + 64));
+    }
+    // number of values <= t (values ascend; the padding is the largest finite value)
+    __device__ __forceinline__ int count_le(float t) const
+    {
+        return (xa.x <= t) + (xa.y <= t) + (xa.z <= t) + (xa.w <= t) + (xb.x <= t) + (xb.y <= t) + (xb.z <= t) + (xb.w <= t);
+    }
+};
+
+// Adds the first n (0..8) elements of a group to (s0, s1[, s2]): the eight terms are summed pairwise,
+// a fixed order with a short dependency chain.  Elements past n are masked before any arithmetic.
+template <bool WANT_C>
+__device__ __forceinline__ void add_group(const Group &grp, int n, double &s0, double &s1, double &s2)
+{
+    const float xs[8] = {grp.xa.x, grp.xa.y, grp.xa.z, grp.xa.w, grp.xb.x, grp.xb.y, grp.xb.z, grp.xb.w};
+    const float gs[8] = {grp.ga.x, grp.ga.y, grp.ga.z, grp.ga.w, grp.gb.x, grp.gb.y, grp.gb.z, grp.gb.w};
+    double t0[8], t1[8], t2[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const bool in = u < n;
+        const double g = (double)(in ? gs[u] : 0.0f), x = (double)xs[u];   // padding values are finite, so 0 * x = 0
+        t0[u] = g;
+        t1[u] = g * x;
+        if (WANT_C) t2[u] = t1[u] * x;
+    }
+    s0 += ((t0[0] + t0[1]) + (t0[2] + t0[3])) + ((t0[4] + t0[5]) + (t0[6] + t0[7]));
+    s1 += ((t1[0] + t1[1]) + (t1[2] + t1[3])) + ((t1[4] + t1[5]) + (t1[6] + t1[7]));
+    if (WANT_C) s2 += ((t2[0] + t2[1]) + (t2[2] + t2[3])) + ((t2[4] + t2[5]) + (t2[6] + t2[7]));
+}
+
+// A window of 16 ascending group-index entries around the previous boundary position (at least 4
+// entries, i.e. 32 elements, on either side), read from shared memory with four independent loads;
+// only when the boundary left it does the search fall back to a binary search of the whole index.
+struct Window {
+    float4 v[4];
+    int ws;
+    __device__ __forceinline__ void load(const float *gi, int ngi, int guess)   // gi: shared memory
+    {
+        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, ngi - WIN));
+        const float4 *p = reinterpret_cast<const float4 *>(gi + ws);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = p[q];
+    }
+    // number of window entries <= t: a 4-step binary search over the 16 ascending registers
+    __device__ __forceinline__ int count_le(float t) const
+    {
+        const bool b3 = v[1].w <= t;                                   // entry 7
+        const float4 h = b3 ? v[3] : v[1], l = b3 ? v[2] : v[0];      // entries 8..15 or 0..7: h = upper four, l = lower four
+        const bool b2 = l.w <= t;                                      // entry 3 of the half
+        const float4 q = b2 ? h : l;
+        const bool b1 = q.y <= t;
+        const float e = b1 ? q.z : q.x;
+        const float e2 = b1 ? q.w : q.y;
+        const bool b0 = e <= t;
+        // position inside the quad: entries <= t among (x, y, z, w)
+        const int inq = b1 ? (b0 ? ((e2 <= t) ? 4 : 3) : 2) : (b0 ? 1 : 0);
+        return (b3 ? 8 : 0) + (b2 ? 4 : 0) + inq;
+    }
+};
+
+// s1 / s0 for s0 > 0: binary32 reciprocal seed and two binary64 Newton corrections (relative
+// error about 2^-60, i.e. the correctly rounded quotient up to the last bit or so); operands far
+// outside the binary32 range take the plain division.
+__device__ __forceinline__ double quotient(double s1, double s0)
+{
+    const float s0f = (float)s0;
+    if (!(s0f > 1e-30f && s0f < 1e30f) || !(fabs(s1) < 1e30)) return s1 / s0;
+    const float rf = __frcp_rn(s0f);
+    const double rd = (double)rf;
+    double q = (double)((float)s1 * rf);
+    q = fma(fma(-q, s0, s1), rd, q);
+    q = fma(fma(-q, s0, s1), rd, q);
+    return q;
+}
+
+// Lloyd iterations and the error table entry of one row, run by ONE warp (all 32 lanes call).
+// Lane L owns centroid L of the row's concatenated centroid record and the boundary above it.
+// Per iteration a lane: forms the exact midpoint; counts the group-index entries below it in the
+// register window (falling back to a binary search of the group index when the boundary left the
+// window); loads that one group record, which gives the exact boundary position (values), the
+// prefix sums at the group start and the few elements in between.
+// On return sm.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
+__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float *gi, int nd, const ClusterArgs &a, int64_t row,
+                                           LloydSmem &sm)
+{
+    const int lane = threadIdx.x & 31;
+    const int m = a.m;
+    const RowRecord R = row_record(m);
+    const unsigned char *groups = rec + R.groups;
+    const double *P2 = reinterpret_cast<const double *>(rec + R.p2);
+    const double *tot = reinterpret_cast<const double *>(rec + 16);
+    const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
+    const float INF = __int_as_float(0x7f800000);
+    int bi = 0, off = 0;
+    while (bi < a.nb && lane >= off + (1 << (a.bmin + bi))) { off += 1 << (a.bmin + bi); ++bi; }
+    const bool in_set = lane < a.sumk;
+    const int width = a.bmin + bi;
+    const int k = 1 << width;
+    const int j = lane - off;
+    const bool wanted = in_set && (!a.row_bits || a.row_bits[row] == width);
+    const bool degenerate = wanted && (nd <= k);      // every value gets its own centroid
+    const bool normal = wanted && !degenerate;
+    const bool has_boundary = wanted && j < k - 1;
+    const bool searches = normal && j < k - 1;
+    float c = 0.0f;
+    if (degenerate) c = sm.dvals[min(j, nd - 1)];
+    if (normal) {
+        const int idx = (int)(((long long)(2 * j + 1) * m) / (2 * k));
+        c = __ldg(reinterpret_cast<const float *>(groups + (size_t)(idx >> 3) * SKIM_GROUP_BYTES) + (idx & 7));
+    }
+    const double tot0 = normal ? tot[0] : 0.0, tot1 = normal ? tot[1] : 0.0;
+
+    int Bprev = -1;
+    float tf = INF;                                   // no boundary above the last centroid
+    double err_j = 0.0;
+    int gprev = -1;                                   // group of the previous boundary position
+    for (int it = 0;; ++it) {
+        const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
+        int B = m, grp_i = 0, cntk = 0;
+        Group grp;
+        if (has_boundary) {
+            // exact midpoint of two binary32 centroids, rounded down to binary32: x <= midpoint
+            // holds for a binary32 x exactly when x <= tf
+            tf = __double2float_rd(0.5 * ((double)c + (double)c_up));
+            if (tf == 0.0f) tf = 0.0f;
+        }
+        if (searches) {
+            int nle = -1;                              // group-index entries <= tf
+            if (gprev >= 0) {
+                Window win;
+                win.load(gi, ngi, gprev + 1);
+                const int cnt = win.count_le(tf);
+                if ((cnt > 0 || win.ws == 0) && cnt < WIN) nle = win.ws + cnt;
+            }
+            if (nle < 0) {
+                int lo = 0, hi = ngi;
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (gi[mid] <= tf) lo = mid + 1; else hi = mid;
+                }
+                nle = lo;
+            }
+            grp_i = max(nle - 1, 0);
+            gprev = grp_i;
+            const unsigned char *gr = groups + (size_t)grp_i * SKIM_GROUP_BYTES;
+            grp.load(gr);
+            cntk = grp.count_le(tf);
+            B = min((grp_i << 3) + cntk, m);
+        }
+        const bool same = __all_sync(0xffffffffu, B == Bprev);
+        const bool final = (it >= a.iters) || same;
+        Bprev = B;
+        double P0 = 0.0, P1 = 0.0, Pc = 0.0;
+        if (normal) {
+            if (searches) {
+                P0 = grp.p.x;
+                P1 = grp.p.y;
+                if (final) {
+                    Pc = __ldg(P2 + grp_i);
+                    add_group<true>(grp, cntk, P0, P1, Pc);
+                } else {
+                    add_group<false>(grp, cntk, P0, P1, Pc);
+                }
+            } else {
+                // the last centroid of a width has no boundary above it: its prefix is the row total
+                P0 = tot0;
+                P1 = tot1;
+                if (final) Pc = tot[2];
+            }
+        }
+        double Q0 = __shfl_up_sync(0xffffffffu, P0, 1);
+        double Q1 = __shfl_up_sync(0xffffffffu, P1, 1);
+        double Qc = final ? __shfl_up_sync(0xffffffffu, Pc, 1) : 0.0;
+        if (j == 0) { Q0 = 0.0; Q1 = 0.0; Qc = 0.0; }
+        const double S0 = P0 - Q0, S1 = P1 - Q1;
+        if (final) {
+            if (normal) {
+                const double cd = (double)c, S2 = Pc - Qc;
+                err_j = fmax(fma(cd, fma(cd, S0, -2.0 * S1), S2), 0.0);
+            }
+            break;
+        }
+        if (normal && S0 > 0.0) c = (float)quotient(S1, S0);
+    }
+    sm.errs[lane] = err_j;
+    sm.tfs[lane] = has_boundary ? tf : INF;
+    __syncwarp();
+    if (wanted) {
+        if (a.centroids) a.centroids[row * a.sumk + lane] = c;
+        if (j == 0 && a.err) {
+            double e = 0.0;
+            for (int u = 0; u < k; ++u) e += sm.errs[lane + u];
+            if (a.row_bits) a.err[row] = (float)e; else a.err[row * a.nb + bi] = (float)e;
+        }
+    }
+}
+
+// Optional labels of the final assignment, in column order (test/diagnostic output).
+__device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, const LloydSmem &sm)
+{
+    const int m = a.m, lane = threadIdx.x & 31;
+    const uint16_t *Wr = a.W + row * a.ld;
+    int only = -1;
+    if (a.row_bits) only = (int)a.row_bits[row] - a.bmin;
+    for (int e = lane; e < m; e += 32) {
+        float x = __half2float(__ushort_as_half(Wr[e]));
+        if (a.rscale) x = __fmul_rn(x, a.rscale[e]);
+        int off = 0;
+        for (int bi = 0; bi < a.nb; ++bi) {
+            const int k = 1 << (a.bmin + bi);
+            if (only < 0 || only == bi) {
+                int code = 0;
+                for (int u = 0; u < k - 1; ++u) code += (sm.tfs[off + u] < x) ? 1 : 0;
+                if (only < 0) a.codes[((int64_t)bi * a.rows + row) * m + e] = (uint8_t)code;
+                else a.codes[row * (int64_t)m + e] = (uint8_t)code;
+            }
+            off += k;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(ClusterArgs a, int rows_in_chunk)
 {
-    __shared__ PhaseSmem ps_all[LLOYD_WARPS];
+    __shared__ LloydSmem sm_all[LLOYD_WARPS];
+    extern __shared__ __align__(16) float gi_all[];      // [LLOYD_WARPS][sk_entries(m)]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int local = blockIdx.x * LLOYD_WARPS + warp;
     if (local >= rows_in_chunk) return;
-    PhaseSmem &ps = ps_all[warp];
+    LloydSmem &sm = sm_all[warp];
     const int64_t row = a.row0 + local;
     const unsigned char *rec = a.scratch + (size_t)local * (size_t)a.rec_stride;
     const int nd = *reinterpret_cast<const int *>(rec);
-    if (lane < 16) ps.dvals[lane] = reinterpret_cast<const float *>(rec + 64)[lane];
+    if (lane < 16) sm.dvals[lane] = reinterpret_cast<const float *>(rec + 64)[lane];
+    // the row's group index, copied once
+    const int nsk = sk_entries(a.m);
+    float *gi = gi_all + (size_t)warp * nsk;
+    {
+        const float4 *src = reinterpret_cast<const float4 *>(rec + row_record(a.m).gi);
+        float4 *dst = reinterpret_cast<float4 *>(gi);
+        for (int i = lane; i < nsk / 4; i += 32) dst[i] = __ldg(src + i);
+    }
     __syncwarp();
-    lloyd_warp<KeyT>(rec, nd, a, row, ps);
+    lloyd_warp(rec, gi, nd, a, row, sm);
     if (!a.codes) return;
     __syncwarp();
-    write_codes(a, row, ps, lane, 32);
+    write_codes(a, row, sm);
 }
 
 }  // namespace
 
-int skim_launch_lloyd(skim_ctx *ctx, const ClusterArgs &args, int64_t rows, int key_bytes)
+int skim_launch_lloyd(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
 {
     const unsigned blocks = (unsigned)((rows + LLOYD_WARPS - 1) / LLOYD_WARPS);
-    if (key_bytes == 2)
-        skim_lloyd_kernel<uint16_t><<<blocks, LLOYD_WARPS * 32, 0, ctx->stream>>>(args, (int)rows);
-    else
-        skim_lloyd_kernel<uint32_t><<<blocks, LLOYD_WARPS * 32, 0, ctx->stream>>>(args, (int)rows);
+    const size_t smem = (size_t)LLOYD_WARPS * sk_entries(args.m) * sizeof(float);
+    static int attr_dev = -1;
+    static size_t attr_smem = 0;
+    if (attr_dev != ctx->device || attr_smem < smem) {
+        SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_dev = ctx->device;
+        attr_smem = smem;
+    }
+    skim_lloyd_kernel<<<blocks, LLOYD_WARPS * 32, smem, ctx->stream>>>(args, (int)rows);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     return SKIM_OK;
