@@ -142,7 +142,6 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
         const int idx = (int)(((long long)(2 * j + 1) * m) / (2 * k));
         c = __ldg(reinterpret_cast<const float *>(groups + (size_t)(idx >> 3) * SKIM_GROUP_BYTES) + (idx & 7));
     }
-    const double tot0 = normal ? tot[0] : 0.0, tot1 = normal ? tot[1] : 0.0;
 
     int Bprev = -1;
     float tf = INF;                                   // no boundary above the last centroid
@@ -197,9 +196,9 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 }
             } else {
                 // the last centroid of a width has no boundary above it: its prefix is the row total
-                P0 = tot0;
-                P1 = tot1;
-                if (final) Pc = tot[2];
+                P0 = __ldg(tot);
+                P1 = __ldg(tot + 1);
+                if (final) Pc = __ldg(tot + 2);
             }
         }
         double Q0 = __shfl_up_sync(0xffffffffu, P0, 1);
