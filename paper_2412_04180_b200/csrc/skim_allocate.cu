@@ -61,21 +61,46 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
             for (int t = 0; t < steps; ++t) {
                 bool live = (i < n);
                 if (live && pass > 0) live = (q[t] >> (shift + 8)) == prefix;
-                const unsigned d = live ? (unsigned)((q[t] >> shift) & 0xffull) : 0xffffffffu;
-                const unsigned peers = __match_any_sync(0xffffffffu, d);
-                if (live && (peers & ((1u << lane) - 1u)) == 0u) atomicAdd(&hist[d], (unsigned)__popc(peers));
+                const unsigned d = live ? (unsigned)((q[t] >> shift) & 0xffull) : 0u;
+                // keys share their leading bytes, so most lanes of a warp hold the same digit: the
+                // first live lane adds the whole group at once, the others (if any) add themselves
+                const unsigned livemask = __ballot_sync(0xffffffffu, live);
+                if (livemask) {
+                    const int leader = __ffs(livemask) - 1;
+                    const unsigned d0 = __shfl_sync(0xffffffffu, d, leader);
+                    const unsigned same = __ballot_sync(0xffffffffu, live && d == d0);
+                    if (lane == leader) atomicAdd(&hist[d0], (unsigned)__popc(same));
+                    if (live && d != d0) atomicAdd(&hist[d], 1u);
+                }
             }
         }
         __syncthreads();
-        if (tid == 0) {
-            long long need = s_need, above = 0;
-            int d = 255;
-            for (; d > 0; --d) {
-                if (above + (long long)hist[d] >= need) break;
-                above += hist[d];
+        if (warp == 0) {
+            // the digit bucket that holds the need-th largest key: suffix sums over the 256 bins
+            const long long need = s_need;
+            unsigned loc[8];
+            long long sum = 0;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { loc[u] = hist[lane * 8 + u]; sum += loc[u]; }
+            long long incl = sum;                       // bins of this lane and of all higher lanes
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const long long v = __shfl_down_sync(0xffffffffu, incl, off);
+                if (lane + off < 32) incl += v;
             }
-            s_need = need - above;
-            s_prefix = (prefix << 8) | (unsigned long long)d;
+            const long long above_lane = incl - sum;    // keys in bins of higher lanes
+            const bool mine = above_lane < need && need <= incl;
+            const unsigned who = __ballot_sync(0xffffffffu, mine);
+            if (mine || (who == 0u && lane == 0)) {
+                long long above = above_lane;
+                int d = 7;
+                for (; d > 0; --d) {
+                    if (above + (long long)loc[d] >= need) break;
+                    above += loc[d];
+                }
+                s_need = need - above;
+                s_prefix = (prefix << 8) | (unsigned long long)(lane * 8 + d);
+            }
         }
         __syncthreads();
     }
