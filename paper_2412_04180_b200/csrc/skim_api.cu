@@ -73,6 +73,7 @@ int skim_create(skim_ctx **out, int device, void *cuda_stream)
     ctx->scaled = false;
     ctx->scale_cols = 0;
     ctx->launches = 0;
+    ctx->copy_ready = false;
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
         delete ctx;
@@ -84,6 +85,12 @@ int skim_create(skim_ctx **out, int device, void *cuda_stream)
 
 int skim_destroy(skim_ctx *ctx)
 {
+    if (ctx && ctx->copy_ready) {
+        DeviceGuard guard(ctx->device);
+        cudaStreamDestroy(ctx->copy_stream);
+        for (int k = 0; k < SKIM_HOST_CHUNKS; ++k) cudaEventDestroy(ctx->copy_done[k]);
+        cudaEventDestroy(ctx->main_idle);
+    }
     delete ctx;
     return SKIM_OK;
 }
@@ -301,10 +308,32 @@ int skim_quantize_matrix_host(skim_ctx *ctx, const uint16_t *W_host, const float
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SKIM_ERR_CUDA;
     cudaStream_t st = ctx->stream;
-    SKIM_CUDA_OK(cudaMemcpyAsync(s.W, W_host, (size_t)rows * cols * 2, cudaMemcpyHostToDevice, st));
-    SKIM_CUDA_OK(cudaMemcpyAsync(s.G, importance_host, (size_t)rows * cols * 4, cudaMemcpyHostToDevice, st));
-    rc = skim_cluster_rows(ctx, s.W, s.G, rows, cols, cols, bit_set, n_bits, iters, s.centroids, nullptr, s.err);
-    if (rc) return rc;
+    if (!ctx->copy_ready) {
+        SKIM_CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        for (int k = 0; k < SKIM_HOST_CHUNKS; ++k)
+            SKIM_CUDA_OK(cudaEventCreateWithFlags(&ctx->copy_done[k], cudaEventDisableTiming));
+        SKIM_CUDA_OK(cudaEventCreateWithFlags(&ctx->main_idle, cudaEventDisableTiming));
+        ctx->copy_ready = true;
+    }
+    // the staging area may still be read by earlier work on the main stream
+    SKIM_CUDA_OK(cudaEventRecord(ctx->main_idle, st));
+    SKIM_CUDA_OK(cudaStreamWaitEvent(ctx->copy_stream, ctx->main_idle, 0));
+    // rows travel in chunks: chunk k is clustered while chunk k+1 is still on the bus
+    const int64_t per = (rows + SKIM_HOST_CHUNKS - 1) / SKIM_HOST_CHUNKS;
+    const int64_t chunk = per < 256 ? (rows < 256 ? rows : 256) : per;
+    int k = 0;
+    for (int64_t r0 = 0; r0 < rows; r0 += chunk, ++k) {
+        const int64_t n = rows - r0 < chunk ? rows - r0 : chunk;
+        SKIM_CUDA_OK(cudaMemcpyAsync(s.W + r0 * cols, W_host + r0 * cols, (size_t)n * cols * 2, cudaMemcpyHostToDevice,
+                                     ctx->copy_stream));
+        SKIM_CUDA_OK(cudaMemcpyAsync(s.G + r0 * cols, importance_host + r0 * cols, (size_t)n * cols * 4,
+                                     cudaMemcpyHostToDevice, ctx->copy_stream));
+        SKIM_CUDA_OK(cudaEventRecord(ctx->copy_done[k], ctx->copy_stream));
+        SKIM_CUDA_OK(cudaStreamWaitEvent(st, ctx->copy_done[k], 0));
+        rc = skim_cluster_rows(ctx, s.W + r0 * cols, s.G + r0 * cols, n, cols, cols, bit_set, n_bits, iters,
+                               s.centroids + r0 * bs.sumk, nullptr, s.err + r0 * n_bits);
+        if (rc) return rc;
+    }
     rc = skim_allocate_bits(ctx, s.err, rows, bit_set, n_bits, budget, s.bits, nullptr);
     if (rc) return rc;
     rc = skim_quantize(ctx, s.W, rows, cols, cols, s.bits, s.centroids, bit_set, n_bits, s.packed, s.row_order,

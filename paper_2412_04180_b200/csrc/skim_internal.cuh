@@ -8,6 +8,7 @@
 #include "skim.h"
 
 #define SKIM_MAX_NBITS SKIM_MAX_BIT
+#define SKIM_HOST_CHUNKS 8   // row chunks of the host-buffer entry point
 #define SKIM_MAX_SUMK 30  // 2 + 4 + 8 + 16: one warp lane per centroid
 
 struct skim_ctx {
@@ -20,6 +21,12 @@ struct skim_ctx {
     bool scaled;          // a scale vector is installed
     int64_t scale_cols;
     int64_t launches;
+    // host-buffer entry point: a second stream for the host-to-device copies, so that the copy
+    // of one row chunk runs under the clustering of the previous one (created on first use)
+    cudaStream_t copy_stream;
+    cudaEvent_t copy_done[SKIM_HOST_CHUNKS];
+    cudaEvent_t main_idle;
+    bool copy_ready;
 };
 
 // Workspace layout (all offsets 256-byte aligned), carved per call for the call's (rows, cols).

@@ -4,8 +4,9 @@
 //
 //   skim_rank_rows_kernel  one block: stable partition of the rows by width -> packed position of
 //                          every row, row order, group starts and word offsets.
-//   skim_pack_kernel       one block per row: label = number of midpoints below the element
-//                          (4-step search over <= 15 boundaries), 8 labels per thread, four
+//   skim_pack_kernel       one block per row: label = number of midpoints below the element,
+//                          8 labels per thread (packed fp16 compares, two weights per instruction,
+//                          when no scale is installed; a 4-step search in binary32 otherwise), four
 //                          threads merge their bit fields with shuffles and store whole words.
 #include "skim_internal.cuh"
 
@@ -104,9 +105,32 @@ struct PackArgs {
     uint16_t *lut;
 };
 
+// Labels of 8 fp16 weights (no scale installed) with packed half-precision compares: a weight is
+// above a boundary exactly when it is above the boundary rounded down to fp16, so two weights are
+// compared per instruction and the label is the running sum of the 0/1 results.  Returns the 8
+// labels as B-bit fields.
+template <int B>
+__device__ __forceinline__ uint32_t labels8_half(const uint4 raw, const __half2 *th)
+{
+    const __half2 *p = reinterpret_cast<const __half2 *>(&raw);
+    const __half2 magic = __floats2half2_rn(1024.0f, 1024.0f);   // 1024 + n has n in its low mantissa bits
+    uint32_t v = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        __half2 cnt = magic;
+#pragma unroll
+        for (int j = 0; j < (1 << B) - 1; ++j) cnt = __hadd2(cnt, __hgt2(p[u], th[j]));
+        const uint32_t bits = *reinterpret_cast<const uint32_t *>(&cnt);
+        v |= (bits & 0xfu) << ((2 * u) * B);
+        v |= ((bits >> 16) & 0xfu) << ((2 * u + 1) * B);
+    }
+    return v;
+}
+
 __global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
 {
     __shared__ float tf[16];
+    __shared__ __half2 th_s[16];
     const int tid = threadIdx.x;
     const int64_t row = blockIdx.x;
     const int pos = a.row_pos[row];
@@ -126,8 +150,12 @@ __global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
             if (t == 0.0f) t = 0.0f;
         }
         tf[tid] = t;
+        th_s[tid] = __half2half2(__float2half_rd(t));
     }
     __syncthreads();
+    __half2 th[15];
+#pragma unroll
+    for (int j = 0; j < 15; ++j) th[j] = th_s[j];
     const int64_t stride = skim_row_stride_words(a.cols, b);
     uint32_t *dst = a.packed + a.group_info[a.nb + 1 + bi] + (int64_t)(pos - a.group_info[bi]) * stride;
     const int ngroups = (int)((stride + b - 1) / b);   // a group: 32 elements -> b words
@@ -136,44 +164,52 @@ __global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
     for (int base = 0; base < ngroups; base += PT / 4) {
         const int grp = base + quad;
         const int e0 = grp * 32 + ql * 8;
-        float x[8];
-        if (a.vec_ok && e0 + 8 <= a.cols) {
+        uint32_t v = 0;
+        if (a.vec_ok && !a.rscale && e0 + 8 <= a.cols) {
             const uint4 raw = *reinterpret_cast<const uint4 *>(Wr + e0);
-            const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float2 f = __half22float2(h2[u]);
-                x[2 * u] = f.x;
-                x[2 * u + 1] = f.y;
+            switch (b) {
+            case 1: v = labels8_half<1>(raw, th); break;
+            case 2: v = labels8_half<2>(raw, th); break;
+            case 3: v = labels8_half<3>(raw, th); break;
+            default: v = labels8_half<4>(raw, th); break;
             }
-            if (a.rscale) {
+        } else {
+            float x[8];
+            if (a.vec_ok && e0 + 8 <= a.cols) {
+                const uint4 raw = *reinterpret_cast<const uint4 *>(Wr + e0);
+                const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float2 f = __half22float2(h2[u]);
+                    x[2 * u] = f.x;
+                    x[2 * u + 1] = f.y;
+                }
                 const float4 r0 = *reinterpret_cast<const float4 *>(a.rscale + e0);
                 const float4 r1 = *reinterpret_cast<const float4 *>(a.rscale + e0 + 4);
                 x[0] = __fmul_rn(x[0], r0.x); x[1] = __fmul_rn(x[1], r0.y);
                 x[2] = __fmul_rn(x[2], r0.z); x[3] = __fmul_rn(x[3], r0.w);
                 x[4] = __fmul_rn(x[4], r1.x); x[5] = __fmul_rn(x[5], r1.y);
                 x[6] = __fmul_rn(x[6], r1.z); x[7] = __fmul_rn(x[7], r1.w);
+            } else {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int e = e0 + u;
+                    float xv = -__int_as_float(0x7f800000);    // past the row: label 0 (zero padding)
+                    if (e < a.cols) {
+                        xv = __half2float(__ushort_as_half(Wr[e]));
+                        if (a.rscale) xv = __fmul_rn(xv, a.rscale[e]);
+                    }
+                    x[u] = xv;
+                }
             }
-        } else {
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int e = e0 + u;
-                float v = -__int_as_float(0x7f800000);    // past the row: label 0 (zero padding)
-                if (e < a.cols) {
-                    v = __half2float(__ushort_as_half(Wr[e]));
-                    if (a.rscale) v = __fmul_rn(v, a.rscale[e]);
-                }
-                x[u] = v;
+                int code = (x[u] > tf[7]) ? 8 : 0;
+                code += (x[u] > tf[code + 3]) ? 4 : 0;
+                code += (x[u] > tf[code + 1]) ? 2 : 0;
+                code += (x[u] > tf[code]) ? 1 : 0;
+                v |= (uint32_t)code << (u * b);
             }
-        }
-        uint32_t v = 0;
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            int code = (x[u] > tf[7]) ? 8 : 0;
-            code += (x[u] > tf[code + 3]) ? 4 : 0;
-            code += (x[u] > tf[code + 1]) ? 2 : 0;
-            code += (x[u] > tf[code]) ? 1 : 0;
-            v |= (uint32_t)code << (u * b);
         }
         const int sh = ql * 8 * b;                           // bit offset inside the group's b words
         unsigned long long lo = 0ull, hi = 0ull;
