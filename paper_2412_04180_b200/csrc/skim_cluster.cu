@@ -17,7 +17,7 @@
 //   2. sort   block-wide LSD radix sort (8-bit digits, warp-private digit counters, ballot-based
 //             stable ranking), exchanging through one shared-memory buffer.  Afterwards every
 //             1-D cluster is a contiguous interval of the sorted row.
-//   3.        distinct count, group index, block prefix sums (skim_cluster_phases.cuh), row record.
+//   3.        one pass over the sorted row writes its row record (skim_cluster_phases.cuh).
 #include "skim_cluster_phases.cuh"
 
 namespace {
@@ -36,17 +36,14 @@ struct SmemLayout {
     size_t keys, gs, uni, dbase, phase, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nwarps, int blk_shift)
+__host__ __device__ inline SmemLayout smem_layout(int cap, int key_bytes, int nwarps)
 {
     SmemLayout L;
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += (b + 15) & ~(size_t)15; return o; };
     L.keys = take((size_t)cap * key_bytes);
     L.gs = take((size_t)cap * 4);
-    size_t counters = (size_t)nwarps * RADIX * 4;
-    size_t nblk = ((size_t)cap >> blk_shift) + 2;
-    size_t prefix = 3 * nblk * 8;
-    L.uni = take(counters > prefix ? counters : prefix);
+    L.uni = take((size_t)nwarps * RADIX * 4);
     L.dbase = take(RADIX * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.total = off;
@@ -61,11 +58,10 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
     constexpr int NW = THREADS / 32;
     constexpr int CAP = THREADS * ITEMS;
     extern __shared__ __align__(16) unsigned char smem[];
-    const SmemLayout L = smem_layout(CAP, (int)sizeof(KeyT), NW, a.blk_shift);
+    const SmemLayout L = smem_layout(CAP, (int)sizeof(KeyT), NW);
     KeyT *skeys = reinterpret_cast<KeyT *>(smem + L.keys);
     float *sg = reinterpret_cast<float *>(smem + L.gs);
     uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + L.uni);
-    double *PB = reinterpret_cast<double *>(smem + L.uni);
     uint32_t *dbase = reinterpret_cast<uint32_t *>(smem + L.dbase);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
 
@@ -178,16 +174,14 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
         }
     }
 
-    // ---------------------------------------------------------------- 3. distinct count, prefix sums
+    // ---------------------------------------------------------------- 3. row record for the Lloyd kernel
     if (tid == 0) { ps.misc[0] = 0; ps.misc[1] = 0; }
     __syncthreads();
-    count_distinct<KeyT, THREADS>(skeys, m, ps);
-    block_prefix_sums<KeyT, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
-    const int nd = ps.misc[0];
-    if (nd <= 16) collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
-
-    // ---------------------------------------------------------------- 4. row record for the Lloyd kernel
-    write_row_record<KeyT, THREADS>(a, skeys, sg, PB, nd, ps.dvals);
+    const int nd = write_row_record<KeyT, THREADS>(a, skeys, sg, ps);
+    if (nd <= 16) {
+        collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
+        write_distinct_values(a, nd, ps.dvals);
+    }
 }
 
 struct Variant {
@@ -211,15 +205,13 @@ const Variant kVariants16[] = {
 };
 constexpr int kNumVariants = 7;
 
-// Picks the smallest variant that holds `cols` and a prefix block length that fits shared memory.
-const Variant *pick_variant(const Variant *table, int64_t cols, int max_smem, int *blk_shift, size_t *smem)
+// Picks the smallest variant that holds `cols` and fits shared memory.
+const Variant *pick_variant(const Variant *table, int64_t cols, int max_smem, size_t *smem)
 {
     for (int v = 0; v < kNumVariants; ++v) {
         if (table[v].cap < cols) continue;
-        for (int s = 3; s <= 5; ++s) {
-            const SmemLayout L = smem_layout(table[v].cap, table[v].key_bytes, table[v].threads / 32, s);
-            if (L.total <= (size_t)max_smem) { *blk_shift = s; *smem = L.total; return &table[v]; }
-        }
+        const SmemLayout L = smem_layout(table[v].cap, table[v].key_bytes, table[v].threads / 32);
+        if (L.total <= (size_t)max_smem) { *smem = L.total; return &table[v]; }
     }
     return nullptr;
 }
@@ -230,8 +222,8 @@ int skim_cluster_max_cols(int max_smem_optin, int64_t *out)
 {
     int64_t best = 0;
     for (int v = 0; v < kNumVariants; ++v) {
-        int s; size_t b;
-        if (pick_variant(kVariants32, kVariants32[v].cap, max_smem_optin, &s, &b)) best = kVariants32[v].cap;
+        size_t b;
+        if (pick_variant(kVariants32, kVariants32[v].cap, max_smem_optin, &b)) best = kVariants32[v].cap;
     }
     *out = best;
     return SKIM_OK;
@@ -256,7 +248,6 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     a.bmin = bits.b_min;
     a.sumk = bits.sumk;
     a.iters = iters;
-    a.blk_shift = 3;
     a.centroids = centroids;
     a.codes = codes;
     a.err = err;
@@ -270,10 +261,8 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     const Variant *v = nullptr;
     size_t smem = 0;
     if (!fast) {
-        int blk_shift = 3;
-        v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &blk_shift, &smem);
+        v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &smem);
         if (!v) return SKIM_ERR_SHAPE;
-        a.blk_shift = blk_shift;
         a.rec_stride = (long long)row_record(a.m).total;
         SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }

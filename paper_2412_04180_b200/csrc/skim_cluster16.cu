@@ -13,11 +13,11 @@
 //   pass 1  high 6 key bits, stable: lanes holding the same digit are found with 6 ballots.
 //   gather  importance is brought into sorted order through the column index; keys and sorted
 //           importance take over the sort buffers, the block prefix sums the rest.
-//   then    block prefix sums (skim_cluster_phases.cuh); the sorted row, its group index and the
-//           prefix sums are written to the row record in global memory, from which the Lloyd
-//           kernel (skim_lloyd.cu) iterates with one warp per row.
+//   then    one pass over the sorted row (skim_cluster_phases.cuh) writes its row record -- group
+//           records with prefix sums, group index, segment table -- to global memory, from which
+//           the Lloyd kernel (skim_lloyd.cu) iterates with one warp per row.
 //
-// Shared memory per 11 008-column row is about 110 KB and the kernel is held to 64 registers, so two
+// Shared memory per 11 008-column row is about 107 KB and the kernel is held to 64 registers, so two
 // rows are resident per SM.
 #include "skim_cluster_phases.cuh"
 
@@ -34,20 +34,16 @@ struct Layout16 {
 };
 
 // buf:  CAP words: packed items during the sort, sorted importance (fp32) afterwards
-// graw: CAP floats: the raw importance row; afterwards keys (first CAP*2 bytes) and the start of PB
-// uni:  pass counters during the sort; the rest of PB afterwards
-__host__ __device__ inline Layout16 layout16(int cap, int nwarps, int blk_shift)
+// graw: CAP floats: the raw importance row; afterwards the sorted keys (first CAP*2 bytes)
+// uni:  pass counters
+__host__ __device__ inline Layout16 layout16(int cap, int nwarps)
 {
     Layout16 L;
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += (b + 15) & ~(size_t)15; return o; };
     L.buf = take((size_t)cap * 4);
     L.graw = take((size_t)cap * 4);
-    const size_t counters = (size_t)D0 * 4 + (size_t)nwarps * D1 * 4;
-    const size_t pb = 3 * 8 * (((size_t)cap >> blk_shift) + 2);
-    const size_t pb_in_graw = (size_t)cap * 2;
-    const size_t pb_over = pb > pb_in_graw ? pb - pb_in_graw : 0;
-    L.uni = take(counters > pb_over ? counters : pb_over);
+    L.uni = take((size_t)D0 * 4 + (size_t)nwarps * D1 * 4);
     L.dbase1 = take(D1 * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.mbar = take(16);
@@ -105,7 +101,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     constexpr int EPT = D0 / THREADS;           // pass-0 counters scanned per thread
     static_assert(D0 % THREADS == 0 && THREADS >= D1, "thread count must divide 1024 and be >= 64");
     extern __shared__ __align__(16) unsigned char smem[];
-    const Layout16 L = layout16(CAP, NW, a.blk_shift);
+    const Layout16 L = layout16(CAP, NW);
     uint32_t *buf = reinterpret_cast<uint32_t *>(smem + L.buf);
     float *graw = reinterpret_cast<float *>(smem + L.graw);
     uint32_t *C0 = reinterpret_cast<uint32_t *>(smem + L.uni);
@@ -113,7 +109,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     uint32_t *dbase1 = reinterpret_cast<uint32_t *>(smem + L.dbase1);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
     uint64_t *mbar = reinterpret_cast<uint64_t *>(smem + L.mbar);
-    uint32_t *scratch = reinterpret_cast<uint32_t *>(ps.wtot);
+    uint32_t *scratch = reinterpret_cast<uint32_t *>(ps.segtot);   // free until the record pass
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = a.m;
@@ -270,17 +266,16 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     __syncthreads();
     uint16_t *skeys = reinterpret_cast<uint16_t *>(graw);
     const float *sg = reinterpret_cast<const float *>(buf);
-    double *PB = reinterpret_cast<double *>(reinterpret_cast<unsigned char *>(graw) + (size_t)CAP * 2);
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) skeys[i * THREADS + tid] = (uint16_t)(item[i] >> 16);
     __syncthreads();
 
-    // ---------------------------------------------------------------- prefix sums, Lloyd, error
-    count_distinct<uint16_t, THREADS>(skeys, m, ps);
-    block_prefix_sums<uint16_t, THREADS>(skeys, sg, m, a.blk_shift, PB, ps);
-    const int nd = ps.misc[0];
-    if (nd <= 16) collect_distinct<uint16_t, THREADS>(skeys, m, nd, ps);
-    write_row_record<uint16_t, THREADS>(a, skeys, sg, PB, nd, ps.dvals);
+    // ---------------------------------------------------------------- row record
+    const int nd = write_row_record<uint16_t, THREADS>(a, skeys, sg, ps);
+    if (nd <= 16) {
+        collect_distinct<uint16_t, THREADS>(skeys, m, nd, ps);
+        write_distinct_values(a, nd, ps.dvals);
+    }
 }
 
 struct Variant16 {
@@ -308,23 +303,20 @@ int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool laun
     if ((reinterpret_cast<uintptr_t>(args.G) & 15u) || (cols % 4) != 0) return 1;
     for (Variant16 &v : kVariants) {
         if (v.cap < cols) continue;
-        for (int s = 3; s <= 5; ++s) {
-            const Layout16 L = layout16(v.cap, v.threads / 32, s);
-            if (L.total > (size_t)ctx->max_smem_optin) continue;
-            args.blk_shift = s;
-            args.rec_stride = (long long)row_record(args.m).total;
-            if (!launch) return SKIM_OK;
-            const ClusterArgs a = args;
-            if (v.dev_set != ctx->device || v.smem_set != (int)L.total) {
-                SKIM_CUDA_OK(cudaFuncSetAttribute(v.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
-                v.dev_set = ctx->device;
-                v.smem_set = (int)L.total;
-            }
-            v.kernel<<<(unsigned)rows, v.threads, L.total, ctx->stream>>>(a);
-            SKIM_CUDA_OK(cudaGetLastError());
-            ctx->launches += 1;
-            return SKIM_OK;
+        const Layout16 L = layout16(v.cap, v.threads / 32);
+        if (L.total > (size_t)ctx->max_smem_optin) continue;
+        args.rec_stride = (long long)row_record(args.m).total;
+        if (!launch) return SKIM_OK;
+        const ClusterArgs a = args;
+        if (v.dev_set != ctx->device || v.smem_set != (int)L.total) {
+            SKIM_CUDA_OK(cudaFuncSetAttribute(v.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
+            v.dev_set = ctx->device;
+            v.smem_set = (int)L.total;
         }
+        v.kernel<<<(unsigned)rows, v.threads, L.total, ctx->stream>>>(a);
+        SKIM_CUDA_OK(cudaGetLastError());
+        ctx->launches += 1;
+        return SKIM_OK;
     }
     return 1;
 }

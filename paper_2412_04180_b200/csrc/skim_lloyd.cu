@@ -122,7 +122,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
     const RowRecord R = row_record(m);
     const unsigned char *groups = rec + R.groups;
     const double *P2 = reinterpret_cast<const double *>(rec + R.p2);
-    const double *tot = reinterpret_cast<const double *>(rec + 16);
+    const double4 *seg = reinterpret_cast<const double4 *>(rec + R.seg);   // 32-byte entries; a few hot lines, served by L1
     const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
     const float INF = __int_as_float(0x7f800000);
     int bi = 0, off = 0;
@@ -186,19 +186,21 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
         double P0 = 0.0, P1 = 0.0, Pc = 0.0;
         if (normal) {
             if (searches) {
-                P0 = grp.p.x;
-                P1 = grp.p.y;
+                const double2 sb = __ldg(reinterpret_cast<const double2 *>(seg + (grp_i >> 5)));   // sums of the earlier segments
+                P0 = sb.x + grp.p.x;
+                P1 = sb.y + grp.p.y;
                 if (final) {
-                    Pc = __ldg(P2 + grp_i);
+                    Pc = __ldg(&seg[grp_i >> 5].z) + __ldg(P2 + grp_i);
                     add_group<true>(grp, cntk, P0, P1, Pc);
                 } else {
                     add_group<false>(grp, cntk, P0, P1, Pc);
                 }
             } else {
                 // the last centroid of a width has no boundary above it: its prefix is the row total
-                P0 = __ldg(tot);
-                P1 = __ldg(tot + 1);
-                if (final) Pc = __ldg(tot + 2);
+                const double2 tot = __ldg(reinterpret_cast<const double2 *>(seg + R.nseg));
+                P0 = tot.x;
+                P1 = tot.y;
+                if (final) Pc = __ldg(&seg[R.nseg].z);
             }
         }
         double Q0 = __shfl_up_sync(0xffffffffu, P0, 1);
