@@ -32,13 +32,16 @@ BIT_SET = [1, 2, 3, 4]
 ITERS = 50
 BUDGET = 3.0
 WORKLOAD = "llama7b_down_proj 4096x11008 fp16, importance LogNormal(0,1.5) fp32, bits {1,2,3,4}, 50 iters, budget 3.0"
-# Algorithmic bytes of the dominant (clustering) kernel: fp16 weight + fp32 importance in,
-# 4 errors + 30 centroids (fp32) out per row.
+# Algorithmic bytes of the clustering stage: fp16 weight + fp32 importance in, 4 errors + 30 centroids
+# (fp32) out per row.  The stage is two kernels: the row-sorting kernel (the dominant one) reads
+# the 6 bytes per element; the Lloyd kernel writes the 136 bytes per row.  The row records that
+# pass between them are scratch, not algorithmic bytes.
 CLUSTER_BYTES_PER_ELEMENT = 6
 CLUSTER_BYTES_PER_ROW = 136
-# DRAM traffic of one clustering launch from the committed ncu capture (bytes), or None when
-# the kernel changed since the counters were taken.
-CLUSTER_TRAFFIC_BYTES = 278_339_000   # 2 x (135.56 MB read + 3.61 MB written) of the 2048-row capture in profiles/
+# DRAM traffic of one launch of the dominant kernel per row, from the committed ncu capture
+# (bytes), or None when the kernel changed since the counters were taken.
+SORT_TRAFFIC_BYTES_PER_ROW = None
+DOMINANT_KERNEL = "skim_sort16_kernel"
 
 
 def measured_peak():
@@ -150,7 +153,7 @@ def run_reference(args):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2412_04180_b200 import build
+    from paper_2412_04180_b200 import build, shard
     from paper_2412_04180_b200.skim import Skim
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -165,7 +168,9 @@ def run_ours(args):
         dist.barrier()
 
     # every rank clusters a matrix of its own (independent problems: no data-path collective)
-    w, g = inputs.make_matrix(ROWS, COLS, SEED + rank)
+    mine = shard.assign_matrices([(ROWS, COLS)] * world, world)[rank]
+    assert len(mine) == 1
+    w, g = inputs.make_matrix(ROWS, COLS, shard.matrix_seed(SEED, mine[0]))
     stream = torch.cuda.Stream()
     ctx = Skim(device=local, stream=stream)
     ctx.reserve(ROWS, COLS)
@@ -219,6 +224,7 @@ def run_ours(args):
     busy(0.4)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     launches0 = ctx.launch_count()
+    ctx.kernel_timing(True)      # events around the two clustering kernels, on the same stream
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     start.record(stream)
@@ -228,14 +234,14 @@ def run_ours(args):
     barrier()
     total_ms = start.elapsed_time(end)
     launches = ctx.launch_count() - launches0
+    sort_total, lloyd_total, timed_chunks = ctx.kernel_times()
+    ctx.kernel_timing(False)
+    sort_ms, lloyd_ms = sort_total / max(1, timed_chunks), lloyd_total / max(1, timed_chunks)
     busy(0.4)
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
         clocks["window"] = "0.4 s of the same steps before and after the timed region, plus the region itself"
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    job_rows_per_s, job_rows, total_ms = shard.job_throughput(ROWS * args.steps, total_ms, "cuda")
     ms_step = total_ms / args.steps
     cluster_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     alloc_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
@@ -266,10 +272,7 @@ def run_ours(args):
             ctx.quantize_matrix_host(Wh, Gh, BIT_SET, ITERS, BUDGET, staging, hout)
         torch.cuda.synchronize()
         e2e_ms = 1e3 * (time.perf_counter() - t0) / n_e2e
-        if world > 1:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = shard.max_over_ranks(e2e_ms, "cuda")
         words = int(hout["group_info"][-1].item())
         d2h = ROWS * nb * 4 + ROWS + ROWS * 4 + 2 * (nb + 1) * 8 + ROWS * (1 << BIT_SET[-1]) * 2 + words * 4
         e2e = {"value": world * ROWS / (e2e_ms / 1e3), "unit": "rows/s", "ms_per_step": e2e_ms,
@@ -282,21 +285,25 @@ def run_ours(args):
         return
     peak, peak_kind = measured_peak()
     cluster_bytes = ROWS * COLS * CLUSTER_BYTES_PER_ELEMENT + ROWS * CLUSTER_BYTES_PER_ROW
-    achieved = cluster_bytes / (cluster_ms * 1e-3) / 1e9
+    sort_bytes = ROWS * COLS * CLUSTER_BYTES_PER_ELEMENT
+    achieved = sort_bytes / (sort_ms * 1e-3) / 1e9
     pipeline_bytes = ROWS * COLS * (6 + 2 + BUDGET / 8) + ROWS * 170
     result = {
-        "metric": METRIC, "value": world * ROWS / (ms_step / 1e3), "unit": "rows/s", "n_gpus": world,
+        "metric": METRIC, "value": job_rows_per_s, "unit": "rows/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": WORKLOAD, "rows": ROWS, "cols": COLS, "l2": "inputs 270 MB per step exceed the 126 MB L2",
                    "early_exit": "on (bit-identical)", "parallelism": f"{world} independent matrices"},
         "weights_per_s": world * ROWS * COLS / (ms_step / 1e3),
         "stage_ms": {"cluster": cluster_ms, "allocate": alloc_ms, "quantize": quant_ms},
+        "kernel_ms": {"skim_sort16_kernel": sort_ms, "skim_lloyd_kernel": lloyd_ms, "launches_timed": timed_chunks},
         "pipeline_hbm_frac": pipeline_bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "cluster_stage_hbm_frac": cluster_bytes / (cluster_ms * 1e-3) / 1e9 / peak,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "skim_cluster16_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": DOMINANT_KERNEL, "achieved": achieved, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": CLUSTER_TRAFFIC_BYTES, "algorithmic_bytes": cluster_bytes, "kernel_ms": cluster_ms},
+                     "traffic": SORT_TRAFFIC_BYTES_PER_ROW * ROWS if SORT_TRAFFIC_BYTES_PER_ROW else None,
+                     "algorithmic_bytes": sort_bytes, "kernel_ms": sort_ms},
     }
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline()

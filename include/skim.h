@@ -215,6 +215,19 @@ int skim_get_status(skim_ctx *ctx, uint64_t *flags);
 /* Number of kernel launches the context has issued so far (host counter). */
 int64_t skim_launch_count(const skim_ctx *ctx);
 
+/*
+ * Measurement aid (no counterpart in the paper).  skim_cluster_rows and skim_cluster_rows_at run,
+ * per chunk of rows, a row-sorting kernel followed by a Lloyd kernel (Algorithm 3, first loop
+ * nest).  With timing enabled the context records a CUDA event on its stream before, between and
+ * after the two, for up to 256 chunks; further chunks go untimed.  skim_kernel_timing(ctx, 1)
+ * starts a fresh series (the events are created on the first call; no device memory is involved),
+ * skim_kernel_timing(ctx, 0) stops recording.  skim_kernel_times waits for the last recorded
+ * event and returns the summed durations in milliseconds and the number of chunks they cover
+ * (host pointers, any may be NULL).
+ */
+int skim_kernel_timing(skim_ctx *ctx, int enable);
+int skim_kernel_times(skim_ctx *ctx, double *sort_ms, double *lloyd_ms, int64_t *chunks);
+
 const char *skim_strerror(int code);
 
 #ifdef __cplusplus

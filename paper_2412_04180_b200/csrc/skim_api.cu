@@ -74,6 +74,9 @@ int skim_create(skim_ctx **out, int device, void *cuda_stream)
     ctx->scale_cols = 0;
     ctx->launches = 0;
     ctx->copy_ready = false;
+    ctx->timing = false;
+    ctx->timing_ready = false;
+    ctx->timing_used = 0;
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
         delete ctx;
@@ -90,6 +93,11 @@ int skim_destroy(skim_ctx *ctx)
         cudaStreamDestroy(ctx->copy_stream);
         for (int k = 0; k < SKIM_HOST_CHUNKS; ++k) cudaEventDestroy(ctx->copy_done[k]);
         cudaEventDestroy(ctx->main_idle);
+    }
+    if (ctx && ctx->timing_ready) {
+        DeviceGuard guard(ctx->device);
+        for (int k = 0; k < SKIM_TIMING_SLOTS; ++k)
+            for (int e = 0; e < 3; ++e) cudaEventDestroy(ctx->timing_ev[k][e]);
     }
     delete ctx;
     return SKIM_OK;
@@ -373,6 +381,43 @@ int skim_get_status(skim_ctx *ctx, uint64_t *flags)
 }
 
 int64_t skim_launch_count(const skim_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int skim_kernel_timing(skim_ctx *ctx, int enable)
+{
+    if (!ctx) return SKIM_ERR_NULL;
+    if (enable && !ctx->timing_ready) {
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok) return SKIM_ERR_CUDA;
+        for (int k = 0; k < SKIM_TIMING_SLOTS; ++k)
+            for (int e = 0; e < 3; ++e) SKIM_CUDA_OK(cudaEventCreate(&ctx->timing_ev[k][e]));
+        ctx->timing_ready = true;
+    }
+    ctx->timing = enable != 0;
+    ctx->timing_used = 0;
+    return SKIM_OK;
+}
+
+int skim_kernel_times(skim_ctx *ctx, double *sort_ms, double *lloyd_ms, int64_t *chunks)
+{
+    if (!ctx) return SKIM_ERR_NULL;
+    double s = 0.0, l = 0.0;
+    if (ctx->timing_used > 0) {
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok) return SKIM_ERR_CUDA;
+        SKIM_CUDA_OK(cudaEventSynchronize(ctx->timing_ev[ctx->timing_used - 1][2]));
+        for (int k = 0; k < ctx->timing_used; ++k) {
+            float a = 0.0f, b = 0.0f;
+            SKIM_CUDA_OK(cudaEventElapsedTime(&a, ctx->timing_ev[k][0], ctx->timing_ev[k][1]));
+            SKIM_CUDA_OK(cudaEventElapsedTime(&b, ctx->timing_ev[k][1], ctx->timing_ev[k][2]));
+            s += a;
+            l += b;
+        }
+    }
+    if (sort_ms) *sort_ms = s;
+    if (lloyd_ms) *lloyd_ms = l;
+    if (chunks) *chunks = ctx->timing_used;
+    return SKIM_OK;
+}
 
 const char *skim_strerror(int code)
 {

@@ -271,6 +271,8 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     for (int64_t row0 = 0; row0 < rows; row0 += SKIM_CLUSTER_CHUNK_ROWS) {
         const int64_t n = rows - row0 < SKIM_CLUSTER_CHUNK_ROWS ? rows - row0 : SKIM_CLUSTER_CHUNK_ROWS;
         a.row0 = row0;
+        cudaEvent_t *tev = (ctx->timing && ctx->timing_used < SKIM_TIMING_SLOTS) ? ctx->timing_ev[ctx->timing_used] : nullptr;
+        if (tev) SKIM_CUDA_OK(cudaEventRecord(tev[0], ctx->stream));
         if (fast) {
             const int rc = skim_launch_sort16(ctx, a, n, true);
             if (rc) return rc < 0 ? rc : SKIM_ERR_SHAPE;
@@ -279,8 +281,13 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
             SKIM_CUDA_OK(cudaGetLastError());
             ctx->launches += 1;
         }
+        if (tev) SKIM_CUDA_OK(cudaEventRecord(tev[1], ctx->stream));
         const int rc = skim_launch_lloyd(ctx, a, n);
         if (rc) return rc;
+        if (tev) {
+            SKIM_CUDA_OK(cudaEventRecord(tev[2], ctx->stream));
+            ctx->timing_used += 1;
+        }
     }
     return SKIM_OK;
 }

@@ -10,6 +10,7 @@
 #define SKIM_MAX_NBITS SKIM_MAX_BIT
 #define SKIM_HOST_CHUNKS 8   // row chunks of the host-buffer entry point
 #define SKIM_MAX_SUMK 30  // 2 + 4 + 8 + 16: one warp lane per centroid
+#define SKIM_TIMING_SLOTS 256   // clustering chunks whose kernel times skim_kernel_timing can hold
 
 struct skim_ctx {
     int device;
@@ -27,6 +28,12 @@ struct skim_ctx {
     cudaEvent_t copy_done[SKIM_HOST_CHUNKS];
     cudaEvent_t main_idle;
     bool copy_ready;
+    // optional kernel timing: events before the sort kernel, between the two kernels and after
+    // the Lloyd kernel of every clustering chunk, on the context's stream
+    bool timing;
+    bool timing_ready;
+    int timing_used;
+    cudaEvent_t timing_ev[SKIM_TIMING_SLOTS][3];
 };
 
 // Workspace layout (all offsets 256-byte aligned), carved per call for the call's (rows, cols).

@@ -22,7 +22,8 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
            "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits",
            "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_scale_update", "skim_host_staging_bytes",
-           "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_strerror"]
+           "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
+           "skim_kernel_times", "skim_strerror"]
 
 
 class SkimError(RuntimeError):
@@ -251,6 +252,16 @@ class Skim:
 
     def launch_count(self):
         return int(lib().skim_launch_count(self._h))
+
+    def kernel_timing(self, enable=True):
+        """Starts (or stops) recording CUDA events around the sort and Lloyd kernels of every clustering chunk."""
+        _chk(lib().skim_kernel_timing(self._h, C.c_int(1 if enable else 0)), "skim_kernel_timing")
+
+    def kernel_times(self):
+        """Returns (sort kernel ms, Lloyd kernel ms, chunks) summed since kernel_timing(True); waits for the events."""
+        s, l, n = C.c_double(), C.c_double(), C.c_int64()
+        _chk(lib().skim_kernel_times(self._h, C.byref(s), C.byref(l), C.byref(n)), "skim_kernel_times")
+        return s.value, l.value, n.value
 
 
 STATIC_MAX_ROWS = 65536
