@@ -20,20 +20,34 @@ __device__ __forceinline__ unsigned long long ordered_bits(double v)
     return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// keys of one row: q[t] for t = 0 .. nb-2
+// keys of one row: q[t] for t = 0 .. nb-2 (entries beyond stay 0)
 __device__ __forceinline__ void row_keys(const float *err, int64_t i, int nb, unsigned long long *q)
 {
     double run = 0.0;
-    for (int t = 0; t + 1 < nb; ++t) {
-        const double gain = (double)err[i * nb + t] - (double)err[i * nb + t + 1];
-        run = (t == 0 || gain < run) ? gain : run;
-        q[t] = ordered_bits(run);
+    float prev = __ldg(err + i * nb);
+#pragma unroll
+    for (int t = 0; t < SKIM_MAX_NBITS - 1; ++t) {
+        q[t] = 0ull;
+        if (t + 1 < nb) {
+            const float next = __ldg(err + i * nb + t + 1);
+            const double gain = (double)prev - (double)next;
+            run = (t == 0 || gain < run) ? gain : run;
+            q[t] = ordered_bits(run);
+            prev = next;
+        }
     }
 }
 
+// Rows are dealt to threads so that a warp reads consecutive rows: warp w owns the rows
+// [w * rounds * 32, (w + 1) * rounds * 32), lane l takes row j * 32 + l of that range in round j.
+// CACHE_ROWS > 0: every thread keeps the keys of its (at most CACHE_ROWS) rows in registers for all
+// passes; CACHE_ROWS == 0: keys are recomputed from the table in every pass.
+template <int CACHE_ROWS>
 __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restrict__ err, int64_t n, int nb,
                                                             int bmin, long long K, uint8_t *__restrict__ bits)
 {
+    constexpr int STEPS_MAX = SKIM_MAX_NBITS - 1;
+    constexpr int NC = CACHE_ROWS > 0 ? CACHE_ROWS : 1;
     __shared__ unsigned int hist[256];
     __shared__ unsigned long long s_prefix;
     __shared__ long long s_need;
@@ -45,34 +59,85 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
         for (int64_t i = tid; i < n; i += AT) bits[i] = (uint8_t)bmin;
         return;
     }
+    const int rounds = (int)((n + AT - 1) / AT);
+    const int64_t row_base = (int64_t)warp * rounds * 32 + lane;
+
+    unsigned long long cache[NC][STEPS_MAX];
+    if (CACHE_ROWS > 0) {
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+            const int64_t i = row_base + (int64_t)j * 32;
+            unsigned long long q[SKIM_MAX_NBITS] = {0ull, 0ull, 0ull, 0ull};
+            if (j < rounds && i < n) row_keys(err, i, nb, q);
+#pragma unroll
+            for (int t = 0; t < STEPS_MAX; ++t) cache[j][t] = q[t];
+        }
+    }
+    // keys of this thread's row of round j (valid only when the row exists)
+    auto keys_of = [&](int j, int64_t i, unsigned long long *q) {
+        if (CACHE_ROWS > 0) {
+#pragma unroll
+            for (int jj = 0; jj < NC; ++jj)
+                if (jj == j) {
+#pragma unroll
+                    for (int t = 0; t < STEPS_MAX; ++t) q[t] = cache[jj][t];
+                }
+        } else {
+            row_keys(err, i, nb, q);
+        }
+    };
+
     if (tid == 0) { s_prefix = 0ull; s_need = K; }
+    for (int d = tid; d < 256; d += AT) hist[d] = 0u;
     __syncthreads();
 
     // radix select: after pass p the top 8(p+1) bits of the K-th largest key are known
     for (int pass = 0; pass < 8; ++pass) {
         const int shift = 56 - 8 * pass;
-        for (int d = tid; d < 256; d += AT) hist[d] = 0u;
-        __syncthreads();
         const unsigned long long prefix = s_prefix;
-        for (int64_t base = 0; base < n; base += AT) {
-            const int64_t i = base + tid;
+        // Live keys share their leading bytes, so most of a warp's keys fall into one bin: the warp
+        // settles on the digit of its first live key, every lane counts its keys with that digit
+        // privately, and one atomic per warp adds them all; other digits are added one by one.
+        bool have_digit = false;     // warp-uniform
+        unsigned d0 = 0u;
+        unsigned cnt0 = 0u;
+#pragma unroll 1
+        for (int j = 0; j < rounds; ++j) {
+            const int64_t i = row_base + (int64_t)j * 32;
+            const bool row_ok = i < n;
             unsigned long long q[SKIM_MAX_NBITS];
-            if (i < n) row_keys(err, i, nb, q);
-            for (int t = 0; t < steps; ++t) {
-                bool live = (i < n);
-                if (live && pass > 0) live = (q[t] >> (shift + 8)) == prefix;
-                const unsigned d = live ? (unsigned)((q[t] >> shift) & 0xffull) : 0u;
-                // keys share their leading bytes, so most lanes of a warp hold the same digit: the
-                // first live lane adds the whole group at once, the others (if any) add themselves
-                const unsigned livemask = __ballot_sync(0xffffffffu, live);
-                if (livemask) {
-                    const int leader = __ffs(livemask) - 1;
-                    const unsigned d0 = __shfl_sync(0xffffffffu, d, leader);
-                    const unsigned same = __ballot_sync(0xffffffffu, live && d == d0);
-                    if (lane == leader) atomicAdd(&hist[d0], (unsigned)__popc(same));
-                    if (live && d != d0) atomicAdd(&hist[d], 1u);
+            if (row_ok) keys_of(j, i, q);
+            unsigned dig[STEPS_MAX];
+            bool live[STEPS_MAX];
+            int first = -1;
+#pragma unroll
+            for (int t = 0; t < STEPS_MAX; ++t) {
+                live[t] = row_ok && t < steps && (pass == 0 || (q[t] >> (shift + 8)) == prefix);
+                dig[t] = live[t] ? (unsigned)((q[t] >> shift) & 0xffull) : 0u;
+                if (live[t] && first < 0) first = t;
+            }
+            if (!have_digit) {
+                const unsigned any = __ballot_sync(0xffffffffu, first >= 0);
+                if (any) {
+                    unsigned mine = 0u;
+#pragma unroll
+                    for (int t = 0; t < STEPS_MAX; ++t)
+                        if (t == first) mine = dig[t];
+                    d0 = __shfl_sync(0xffffffffu, mine, __ffs(any) - 1);
+                    have_digit = true;
                 }
             }
+#pragma unroll
+            for (int t = 0; t < STEPS_MAX; ++t) {
+                if (live[t]) {
+                    if (dig[t] == d0) ++cnt0;
+                    else atomicAdd(&hist[dig[t]], 1u);
+                }
+            }
+        }
+        if (have_digit) {
+            const unsigned total = __reduce_add_sync(0xffffffffu, cnt0);
+            if (lane == 0 && total) atomicAdd(&hist[d0], total);
         }
         __syncthreads();
         if (warp == 0) {
@@ -82,6 +147,9 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
             long long sum = 0;
 #pragma unroll
             for (int u = 0; u < 8; ++u) { loc[u] = hist[lane * 8 + u]; sum += loc[u]; }
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < 8; ++u) hist[lane * 8 + u] = 0u;    // ready for the next pass
             long long incl = sum;                       // bins of this lane and of all higher lanes
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
@@ -107,39 +175,57 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
     const unsigned long long thr = s_prefix;   // the K-th largest key
     const long long take_eq = s_need;          // how many items equal to it are taken, in row-major order
 
-    // rank of equal items: every thread owns a contiguous chunk of rows
-    const int64_t per = (n + AT - 1) / AT;
-    const int64_t r0 = min(n, (int64_t)tid * per), r1 = min(n, r0 + per);
-    long long eq = 0;
-    for (int64_t i = r0; i < r1; ++i) {
-        unsigned long long q[SKIM_MAX_NBITS];
-        row_keys(err, i, nb, q);
-        for (int t = 0; t < steps; ++t) eq += (q[t] == thr) ? 1 : 0;
-    }
-    long long inc = eq;
+    // items equal to the threshold are taken in row-major order: count them per warp, ...
+    unsigned eq_all = 0u;
+#pragma unroll 1
+    for (int j = 0; j < rounds; ++j) {
+        const int64_t i = row_base + (int64_t)j * 32;
+        if (i < n) {
+            unsigned long long q[SKIM_MAX_NBITS];
+            keys_of(j, i, q);
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const long long v = __shfl_up_sync(0xffffffffu, inc, off);
-        if (lane >= off) inc += v;
-    }
-    if (lane == 31) wsum[warp] = inc;
-    __syncthreads();
-    long long before = inc - eq;
-    for (int w = 0; w < warp; ++w) before += wsum[w];
-
-    for (int64_t i = r0; i < r1; ++i) {
-        unsigned long long q[SKIM_MAX_NBITS];
-        row_keys(err, i, nb, q);
-        int extra = 0;
-        for (int t = 0; t < steps; ++t) {
-            if (q[t] > thr) {
-                ++extra;
-            } else if (q[t] == thr) {
-                if (before < take_eq) ++extra;
-                ++before;
-            }
+            for (int t = 0; t < STEPS_MAX; ++t) eq_all += (t < steps && q[t] == thr) ? 1u : 0u;
         }
-        bits[i] = (uint8_t)(bmin + extra);
+    }
+    const unsigned warp_eq = __reduce_add_sync(0xffffffffu, eq_all);
+    if (lane == 0) wsum[warp] = (long long)warp_eq;
+    __syncthreads();
+    long long carry = 0;                       // equal items in rows before this warp's current round
+    for (int w = 0; w < warp; ++w) carry += wsum[w];
+
+    // ... then rank them round by round with a warp prefix sum (rows of a round ascend with the lane)
+#pragma unroll 1
+    for (int j = 0; j < rounds; ++j) {
+        const int64_t i = row_base + (int64_t)j * 32;
+        const bool row_ok = i < n;
+        unsigned long long q[SKIM_MAX_NBITS];
+        if (row_ok) keys_of(j, i, q);
+        unsigned eq = 0u;
+#pragma unroll
+        for (int t = 0; t < STEPS_MAX; ++t) eq += (row_ok && t < steps && q[t] == thr) ? 1u : 0u;
+        unsigned inc = eq;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned v = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += v;
+        }
+        long long before = carry + (long long)(inc - eq);
+        carry += (long long)__shfl_sync(0xffffffffu, inc, 31);
+        if (row_ok) {
+            int extra = 0;
+#pragma unroll
+            for (int t = 0; t < STEPS_MAX; ++t) {
+                if (t < steps) {
+                    if (q[t] > thr) {
+                        ++extra;
+                    } else if (q[t] == thr) {
+                        if (before < take_eq) ++extra;
+                        ++before;
+                    }
+                }
+            }
+            bits[i] = (uint8_t)(bmin + extra);
+        }
     }
 }
 
@@ -148,7 +234,10 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
 int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int64_t K,
                          uint8_t *out_bits)
 {
-    skim_allocate_kernel<<<1, AT, 0, ctx->stream>>>(err, rows, bits.n_bits, bits.b_min, (long long)K, out_bits);
+    if (rows <= 4 * AT)
+        skim_allocate_kernel<4><<<1, AT, 0, ctx->stream>>>(err, rows, bits.n_bits, bits.b_min, (long long)K, out_bits);
+    else
+        skim_allocate_kernel<0><<<1, AT, 0, ctx->stream>>>(err, rows, bits.n_bits, bits.b_min, (long long)K, out_bits);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     return SKIM_OK;
