@@ -177,9 +177,10 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
     // ---------------------------------------------------------------- 3. row record for the Lloyd kernel
     if (tid == 0) { ps.misc[0] = 0; ps.misc[1] = 0; }
     __syncthreads();
-    const int nd = write_row_record<KeyT, THREADS>(a, skeys, sg, ps);
+    const SortedArrays<KeyT> src{skeys, sg};
+    const int nd = write_row_record<KeyT, THREADS>(a, src, ps);
     if (nd <= 16) {
-        collect_distinct<KeyT, THREADS>(skeys, m, nd, ps);
+        collect_distinct<KeyT, THREADS>(src, m, nd, ps);
         write_distinct_values(a, nd, ps.dvals);
     }
 }

@@ -11,11 +11,11 @@
 //           loop also builds the per-warp histogram of the next pass (the element's owner warp in
 //           pass 1 follows from its slot).
 //   pass 1  high 6 key bits, stable: lanes holding the same digit are found with 6 ballots.
-//   gather  importance is brought into sorted order through the column index; keys and sorted
-//           importance take over the sort buffers, the block prefix sums the rest.
-//   then    one pass over the sorted row (skim_cluster_phases.cuh) writes its row record -- group
+//   then    one pass over the sorted items (skim_cluster_phases.cuh) writes the row record -- group
 //           records with prefix sums, group index, segment table -- to global memory, from which
-//           the Lloyd kernel (skim_lloyd.cu) iterates with one warp per row.
+//           the Lloyd kernel (skim_lloyd.cu) iterates with one warp per row.  The pass fetches every
+//           element's importance through the column index the item carries, so the importance
+//           row is never rearranged in shared memory.
 //
 // Shared memory per 11 008-column row is about 107 KB and the kernel is held to 64 registers, so two
 // rows are resident per SM.
@@ -33,8 +33,8 @@ struct Layout16 {
     size_t buf, graw, uni, dbase1, phase, mbar, total;
 };
 
-// buf:  CAP words: packed items during the sort, sorted importance (fp32) afterwards
-// graw: CAP floats: the raw importance row; afterwards the sorted keys (first CAP*2 bytes)
+// buf:  CAP words: packed items
+// graw: CAP floats: the raw importance row
 // uni:  pass counters
 __host__ __device__ inline Layout16 layout16(int cap, int nwarps)
 {
@@ -89,6 +89,31 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+
+// The sorted row of this kernel: packed items (key << 16 | column) in sorted order, and the raw
+// importance row, which the record pass reads through the column index.
+struct SortedItems16 {
+    const uint32_t *items;
+    const float *graw;
+    __device__ __forceinline__ unsigned group(int e, int m, uint16_t *ks, float *gs) const
+    {
+        const uint4 a = *reinterpret_cast<const uint4 *>(items + e), b = *reinterpret_cast<const uint4 *>(items + e + 4);
+        const uint32_t it[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        unsigned bad = 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            ks[u] = (uint16_t)(it[u] >> 16);
+            float g = 0.0f;
+            if (e + u < m) {
+                g = graw[it[u] & 0xffffu];
+                if (!(g >= 0.0f) || g > 3.0e38f) bad |= 2u;
+            }
+            gs[u] = g;
+        }
+        return bad;
+    }
+    __device__ __forceinline__ uint16_t key_at(int p) const { return (uint16_t)(items[p] >> 16); }
+};
 
 template <int THREADS, int VEC>
 __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16_kernel(ClusterArgs a)
@@ -237,9 +262,9 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
             buf[dbase1[d] + base + rank] = item[i];
         }
     }
-    __syncthreads();
 
-    // ---------------------------------------------------------------- gather importance into sorted order
+    // ---------------------------------------------------------------- the importance row must have landed
+    // (the vote below is also the barrier that ends pass 1)
     {
         const bool landed = mbar_wait_bounded(mbar, 0);
         if (!__syncthreads_and(landed ? 1 : 0)) {
@@ -249,31 +274,11 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
             return;
         }
     }
-    bad = 0;
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) {
-        const int p = i * THREADS + tid;
-        const uint32_t it = buf[p];
-        float g = 0.0f;
-        if (p < m) {
-            g = graw[it & 0xffffu];
-            if (!(g >= 0.0f) || g > 3.0e38f) bad |= 2u;
-        }
-        buf[p] = __float_as_uint(g);
-        item[i] = it;
-    }
-    if (bad) atomicOr(a.status, (unsigned long long)bad);
-    __syncthreads();
-    uint16_t *skeys = reinterpret_cast<uint16_t *>(graw);
-    const float *sg = reinterpret_cast<const float *>(buf);
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) skeys[i * THREADS + tid] = (uint16_t)(item[i] >> 16);
-    __syncthreads();
-
     // ---------------------------------------------------------------- row record
-    const int nd = write_row_record<uint16_t, THREADS>(a, skeys, sg, ps);
+    const SortedItems16 src{buf, graw};
+    const int nd = write_row_record<uint16_t, THREADS>(a, src, ps);
     if (nd <= 16) {
-        collect_distinct<uint16_t, THREADS>(skeys, m, nd, ps);
+        collect_distinct<uint16_t, THREADS>(src, m, nd, ps);
         write_distinct_values(a, nd, ps.dvals);
     }
 }

@@ -130,6 +130,24 @@ __device__ __forceinline__ void copy16(void *dst, const void *src, size_t bytes)
     for (size_t i = threadIdx.x; i < bytes / 16; i += THREADS) d[i] = s[i];
 }
 
+// The sorted row as the record pass sees it.  A source gives the keys and importances of one group
+// of 8 sorted elements (positions e .. e+7; the caller masks positions >= m), returns status bits
+// for bad importance values it meets, and gives single keys.
+// This one: keys and importance in two shared-memory arrays, padded to whole groups.
+template <typename KeyT> struct SortedArrays {
+    const KeyT *skeys;
+    const float *sg;
+    __device__ __forceinline__ unsigned group(int e, int, KeyT *ks, float *gs) const
+    {
+        KeyOps<KeyT>::load8(skeys + e, ks);
+        const float4 ga = *reinterpret_cast<const float4 *>(sg + e), gb = *reinterpret_cast<const float4 *>(sg + e + 4);
+        gs[0] = ga.x; gs[1] = ga.y; gs[2] = ga.z; gs[3] = ga.w;
+        gs[4] = gb.x; gs[5] = gb.y; gs[6] = gb.z; gs[7] = gb.w;
+        return 0u;
+    }
+    __device__ __forceinline__ KeyT key_at(int p) const { return skeys[p]; }
+};
+
 // Small per-block scratch of the phases below.
 struct PhaseSmem {
     double segtot[96][3];   // sums of every segment of 32 groups (rows of up to 24 576 elements)
@@ -139,11 +157,11 @@ struct PhaseSmem {
 };
 
 // Rare path: the row has nd <= 16 distinct values; stores them ascending in ps.dvals.
-template <typename KeyT, int THREADS>
-__device__ __forceinline__ void collect_distinct(const KeyT *skeys, int m, int nd, PhaseSmem &ps)
+template <typename KeyT, int THREADS, typename Src>
+__device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, PhaseSmem &ps)
 {
     for (int p = threadIdx.x; p < m; p += THREADS) {
-        if (p == 0 || skeys[p] != skeys[p - 1]) {
+        if (p == 0 || src.key_at(p) != src.key_at(p - 1)) {
             const int slot = atomicAdd(&ps.misc[1], 1);
             if (slot < 16) ps.tfs[slot] = __int_as_float(p);
         }
@@ -155,7 +173,7 @@ __device__ __forceinline__ void collect_distinct(const KeyT *skeys, int m, int n
         int rank = 0;
         for (int u = 0; u < nd; ++u) rank += (__shfl_sync(0xffffffffu, p, u) < p) ? 1 : 0;
         __syncwarp();
-        if (lane < nd) ps.dvals[rank] = KeyOps<KeyT>::to_float(skeys[p]);
+        if (lane < nd) ps.dvals[rank] = KeyOps<KeyT>::to_float(src.key_at(p));
     }
     __syncthreads();
 }
@@ -167,8 +185,8 @@ __device__ __forceinline__ void collect_distinct(const KeyT *skeys, int m, int n
 // independent, so no warp waits for another.  The same pass counts the row's distinct values.
 // Afterwards one warp turns the segment sums into the segment table.  Call with all threads;
 // ps.misc[0..1] must have been zeroed before (and synced).  Returns nd (distinct values).
-template <typename KeyT, int THREADS>
-__device__ __forceinline__ int write_row_record(const ClusterArgs &a, const KeyT *skeys, const float *sg, PhaseSmem &ps)
+template <typename KeyT, int THREADS, typename Src>
+__device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src &src, PhaseSmem &ps)
 {
     constexpr int NW = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -178,6 +196,7 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const KeyT
     double *p2 = reinterpret_cast<double *>(rec + R.p2);
     float *gi = reinterpret_cast<float *>(rec + R.gi);
     int distinct = 0;
+    unsigned bad = 0u;
     for (int sgm = warp; sgm < R.nseg; sgm += NW) {
         const int q = (sgm << 5) + lane;
         double v0 = 0.0, v1 = 0.0, v2 = 0.0;
@@ -186,10 +205,11 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const KeyT
         if (q < R.ngrp) {
             const int e = q << 3;
             KeyT ks[8];
-            KeyOps<KeyT>::load8(skeys + e, ks);
-            ga = *reinterpret_cast<const float4 *>(sg + e);
-            gb = *reinterpret_cast<const float4 *>(sg + e + 4);
-            KeyT prev = e > 0 ? skeys[e - 1] : (KeyT)0;
+            float gs[8];
+            bad |= src.group(e, m, ks, gs);
+            ga = make_float4(gs[0], gs[1], gs[2], gs[3]);
+            gb = make_float4(gs[4], gs[5], gs[6], gs[7]);
+            KeyT prev = e > 0 ? src.key_at(e - 1) : (KeyT)0;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const bool real = e + u < m;
@@ -197,7 +217,6 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const KeyT
                 distinct += (real && (e + u == 0 || ks[u] != prev)) ? 1 : 0;
                 prev = ks[u];
             }
-            const float gs[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
             double t0[8], t1[8], t2[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -234,6 +253,7 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const KeyT
 #pragma unroll
     for (int off = 16; off; off >>= 1) distinct += __shfl_xor_sync(0xffffffffu, distinct, off);
     if (lane == 0 && distinct) atomicAdd(&ps.misc[0], distinct);
+    if (bad) atomicOr(a.status, (unsigned long long)bad);
     for (int q = R.ngrp + threadIdx.x; q < sk_entries(m); q += THREADS) gi[q] = SKIM_PAD_VALUE;
     __syncthreads();
     const int nd = ps.misc[0];
