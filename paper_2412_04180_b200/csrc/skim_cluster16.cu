@@ -4,20 +4,25 @@
 // With no scale the clustered value IS the fp16 weight, so a 16-bit order-preserving key is exact
 // and the sort moves one 32-bit word per element: (key << 16) | column.
 //
-//   load    128-bit loads of the fp16 row straight into keys; the fp32 importance row is fetched
-//           by one bulk asynchronous copy (cp.async.bulk + mbarrier) that runs under the sort.
-//   pass 0  low 10 key bits, 1024 block-wide counters, slots claimed with shared-memory atomics.
-//           The first pass of an LSD sort need not be stable, so no ranking is needed; the same
-//           loop also builds the per-warp histogram of the next pass (the element's owner warp in
-//           pass 1 follows from its slot).
-//   pass 1  high 6 key bits, stable: lanes holding the same digit are found with 6 ballots.
+//   load    128-bit loads of the fp16 row straight into keys.
+//   pass 0  low 12 key bits, 4096 block-wide counters, slots claimed with shared-memory atomics.
+//           The first pass of an LSD sort need not be stable, so no ranking is needed.  The
+//           scatter also counts, per owner thread of pass 1 and high digit, how many items land
+//           in that thread's stretch of positions.
+//   pass 1  high 4 key bits, stable without any warp-wide ranking: a thread owns a contiguous
+//           stretch of positions, takes its items in position order and numbers them with
+//           counters of its own (one 16-bit counter per thread and digit, prefix-summed across
+//           threads per digit), so the order inside a digit is the order of pass 0.
 //   then    one pass over the sorted items (skim_cluster_phases.cuh) writes the row record -- group
 //           records with prefix sums, group index, segment table -- to global memory, from which
 //           the Lloyd kernel (skim_lloyd.cu) iterates with one warp per row.  The pass fetches every
 //           element's importance through the column index the item carries, so the importance
 //           row is never rearranged in shared memory.
+// The fp32 importance row is fetched by one bulk asynchronous copy (cp.async.bulk + mbarrier) that
+// is issued once pass 0 is over (its landing area holds the pass-0 counters until then) and runs
+// under pass 1.
 //
-// Shared memory per 11 008-column row is about 107 KB and the kernel is held to 64 registers, so two
+// Shared memory per 11 008-column row is about 105 KB and the kernel is held to 64 registers, so two
 // rows are resident per SM.
 #include "skim_cluster_phases.cuh"
 
@@ -25,25 +30,28 @@ namespace {
 
 using namespace skimk;
 
-constexpr int D0_BITS = 10, D0 = 1 << D0_BITS;
-constexpr int D1_BITS = 6, D1 = 1 << D1_BITS;
+constexpr int D0_BITS = 12, D0 = 1 << D0_BITS;
+constexpr int D1_BITS = 4, D1 = 1 << D1_BITS;
 constexpr int MBAR_SPIN_LIMIT = 1 << 22;
+constexpr uint32_t NO_ITEM = 0xffffffffu;    // slot of a thread beyond the row's end (no column is 65 535)
+constexpr uint32_t PAD_ITEM = 0xffff0000u;   // largest key, column 0: fills the last group of the sorted row
 
 struct Layout16 {
-    size_t buf, graw, uni, dbase1, phase, mbar, total;
+    size_t buf, graw, cnt1, dbase1, phase, mbar, total;
 };
 
-// buf:  CAP words: packed items
-// graw: CAP floats: the raw importance row
-// uni:  pass counters
-__host__ __device__ inline Layout16 layout16(int cap, int nwarps)
+// buf:   the packed items, padded to a whole group of 8
+// graw:  the raw importance row; the pass-0 counters (D0 words) until the copy is issued
+// cnt1:  pass-1 counters, [D1][threads] 16-bit
+__host__ __device__ inline Layout16 layout16(int m, int threads)
 {
     Layout16 L;
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += (b + 15) & ~(size_t)15; return o; };
-    L.buf = take((size_t)cap * 4);
-    L.graw = take((size_t)cap * 4);
-    L.uni = take((size_t)D0 * 4 + (size_t)nwarps * D1 * 4);
+    const size_t row = ((size_t)m + 7) / 8 * 8 * 4;
+    L.buf = take(row);
+    L.graw = take(row > (size_t)D0 * 4 ? row : (size_t)D0 * 4);
+    L.cnt1 = take((size_t)D1 * threads * 2);
     L.dbase1 = take(D1 * 4);
     L.phase = take(sizeof(PhaseSmem));
     L.mbar = take(16);
@@ -120,43 +128,39 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
 {
     using K = KeyOps<uint16_t>;
     constexpr int ITEMS = VEC * 8;
-    constexpr int CAP = THREADS * ITEMS;
-    constexpr int NW = THREADS / 32;
-    constexpr int WCHUNK = ITEMS * 32;          // positions owned by one warp in pass 1
     constexpr int EPT = D0 / THREADS;           // pass-0 counters scanned per thread
-    static_assert(D0 % THREADS == 0 && THREADS >= D1, "thread count must divide 1024 and be >= 64");
+    constexpr int WPL = THREADS / 64;           // pass-1 counter words (two counters each) scanned per lane
+    constexpr int NW = THREADS / 32;
+    static_assert(D0 % THREADS == 0 && THREADS % 64 == 0, "thread count must divide 4096 and be a multiple of 64");
     extern __shared__ __align__(16) unsigned char smem[];
-    const Layout16 L = layout16(CAP, NW);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m = a.m;
+    const int mpad = (m + 7) & ~7;
+    const Layout16 L = layout16(m, THREADS);
     uint32_t *buf = reinterpret_cast<uint32_t *>(smem + L.buf);
     float *graw = reinterpret_cast<float *>(smem + L.graw);
-    uint32_t *C0 = reinterpret_cast<uint32_t *>(smem + L.uni);
-    uint32_t *cnt1 = C0 + D0;
+    uint32_t *C0 = reinterpret_cast<uint32_t *>(smem + L.graw);
+    uint32_t *cnt1w = reinterpret_cast<uint32_t *>(smem + L.cnt1);
+    uint16_t *cnt1 = reinterpret_cast<uint16_t *>(smem + L.cnt1);
     uint32_t *dbase1 = reinterpret_cast<uint32_t *>(smem + L.dbase1);
     PhaseSmem &ps = *reinterpret_cast<PhaseSmem *>(smem + L.phase);
     uint64_t *mbar = reinterpret_cast<uint64_t *>(smem + L.mbar);
     uint32_t *scratch = reinterpret_cast<uint32_t *>(ps.segtot);   // free until the record pass
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int m = a.m;
     const int64_t row = a.row0 + blockIdx.x;
     const uint16_t *Wr = a.W + row * a.ld;
     const float *Gr = a.G + row * a.ld;
 
-    // ---------------------------------------------------------------- set-up, importance row in flight
+    // ---------------------------------------------------------------- set-up
     if (tid == 0) {
         mbar_init(mbar, 1);
         ps.misc[0] = 0;
         ps.misc[1] = 0;
     }
-    for (int d = tid; d < D0 + NW * D1; d += THREADS) C0[d] = 0u;
+    for (int d = tid; d < D0; d += THREADS) C0[d] = 0u;
+    for (int d = tid; d < D1 * THREADS / 2; d += THREADS) cnt1w[d] = 0u;
+    if (tid < mpad - m) buf[m + tid] = PAD_ITEM;
     __syncthreads();
-    if (tid == 0) {
-        const uint32_t bytes = (uint32_t)m * 4u;
-        mbar_expect_tx(mbar, bytes);
-        for (uint32_t o = 0; o < bytes; o += 32768u)
-            bulk_load(reinterpret_cast<unsigned char *>(graw) + o, reinterpret_cast<const unsigned char *>(Gr) + o,
-                      min(32768u, bytes - o), mbar);
-    }
 
     // ---------------------------------------------------------------- load, keys, pass-0 histogram
     uint32_t item[ITEMS];
@@ -171,8 +175,8 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         } else {
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const uint32_t lo = (e0 + 2 * u < m) ? Wr[e0 + 2 * u] : 0x7fffu;         // 0x7fff -> key 0xffff (padding)
-                const uint32_t hi = (e0 + 2 * u + 1 < m) ? Wr[e0 + 2 * u + 1] : 0x7fffu;
+                const uint32_t lo = (e0 + 2 * u < m) ? Wr[e0 + 2 * u] : 0u;
+                const uint32_t hi = (e0 + 2 * u + 1 < m) ? Wr[e0 + 2 * u + 1] : 0u;
                 w[u] = lo | (hi << 16);
             }
         }
@@ -182,9 +186,9 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
             const bool real = e0 + u < m;
             if (real && (h & 0x7c00u) == 0x7c00u) bad |= 1u;
             if (h == 0x8000u) h = 0;                      // -0 and +0 are one value
-            const uint32_t key = real ? (uint32_t)K::from_half_bits(h) : 0xffffu;
-            item[j * 8 + u] = (key << 16) | (uint32_t)(real ? e0 + u : 0);
-            atomicAdd(&C0[key & (D0 - 1)], 1u);
+            const uint32_t key = (uint32_t)K::from_half_bits(h);
+            item[j * 8 + u] = real ? ((key << 16) | (uint32_t)(e0 + u)) : NO_ITEM;
+            if (real) atomicAdd(&C0[key & (D0 - 1)], 1u);
         }
     }
     if (bad) atomicOr(a.status, (unsigned long long)bad);
@@ -211,55 +215,79 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
-        const uint32_t key = item[i] >> 16;
-        const uint32_t pos = atomicAdd(&C0[key & (D0 - 1)], 1u);
-        buf[pos] = item[i];
-        atomicAdd(&cnt1[(pos / WCHUNK) * D1 + (key >> D0_BITS)], 1u);
-    }
-    __syncthreads();
-
-    // ---------------------------------------------------------------- pass 1: scan, stable rank, scatter
-    if (tid < D1) {
-        uint32_t run = 0;
-        for (int w = 0; w < NW; ++w) {
-            const uint32_t c = cnt1[w * D1 + tid];
-            cnt1[w * D1 + tid] = run;
-            run += c;
+        if (item[i] != NO_ITEM) {
+            const uint32_t key = item[i] >> 16;
+            const uint32_t pos = atomicAdd(&C0[key & (D0 - 1)], 1u);
+            buf[pos] = item[i];
+            // one more item of digit key >> 12 in the stretch of pass-1 owner pos / ITEMS
+            const uint32_t owner = pos / ITEMS;
+            atomicAdd(&cnt1w[((key >> D0_BITS) * THREADS + owner) >> 1], (owner & 1u) ? 0x10000u : 1u);
         }
-        // exclusive scan of the 64 digit totals by the first two warps
-        uint32_t inc = run;
+    }
+    // the pass-0 counters are dead: their place takes the importance row, by the asynchronous proxy
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    if (tid == 0) {
+        const uint32_t bytes = (uint32_t)m * 4u;
+        mbar_expect_tx(mbar, bytes);
+        for (uint32_t o = 0; o < bytes; o += 32768u)
+            bulk_load(reinterpret_cast<unsigned char *>(graw) + o, reinterpret_cast<const unsigned char *>(Gr) + o,
+                      min(32768u, bytes - o), mbar);
+    }
+
+    // ---------------------------------------------------------------- pass 1: counters -> positions
+    // per digit, an exclusive prefix sum over the owner threads (a lane takes 2 * WPL consecutive owners)
+    for (int d = warp; d < D1; d += NW) {
+        uint32_t *cw = cnt1w + (d * THREADS) / 2 + lane * WPL;
+        uint32_t wv[WPL], s = 0;
+#pragma unroll
+        for (int u = 0; u < WPL; ++u) { wv[u] = cw[u]; s += (wv[u] & 0xffffu) + (wv[u] >> 16); }
+        uint32_t inc = s;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const uint32_t t = __shfl_up_sync(0xffffffffu, inc, off);
             if (lane >= off) inc += t;
         }
-        if (tid == 31) scratch[0] = inc;
-        __syncwarp();
-        dbase1[tid] = inc - run;
+        if (lane == 31) dbase1[d] = inc;          // the digit's total
+        uint32_t run = inc - s;
+#pragma unroll
+        for (int u = 0; u < WPL; ++u) {
+            const uint32_t lo = wv[u] & 0xffffu, hi = wv[u] >> 16;
+            cw[u] = run | ((run + lo) << 16);
+            run += lo + hi;
+        }
     }
+    // my stretch of positions, in order
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) item[i] = buf[warp * WCHUNK + i * 32 + lane];
+    for (int i = 0; i < ITEMS; i += 4) {
+        const int p = tid * ITEMS + i;
+        uint4 v = make_uint4(NO_ITEM, NO_ITEM, NO_ITEM, NO_ITEM);
+        if (p < m) v = *reinterpret_cast<const uint4 *>(buf + p);     // m is a multiple of 4 here
+        item[i] = v.x; item[i + 1] = v.y; item[i + 2] = v.z; item[i + 3] = v.w;
+    }
     __syncthreads();
-    if (tid >= 32 && tid < D1) dbase1[tid] += scratch[0];
+    if (warp == 0) {
+        // digit totals -> digit bases
+        const uint32_t tot = lane < D1 ? dbase1[lane] : 0u;
+        uint32_t inc = tot;
+#pragma unroll
+        for (int off = 1; off < D1; off <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += t;
+        }
+        if (lane < D1) dbase1[lane] = inc - tot;
+    }
     __syncthreads();
-    {
-        const unsigned lt_mask = (1u << lane) - 1u;
+    // positions = digit base + prefix over the owners before me; then number my items in order
+#pragma unroll 4
+    for (int d = 0; d < D1; ++d) cnt1[d * THREADS + tid] = (uint16_t)(cnt1[d * THREADS + tid] + dbase1[d]);
 #pragma unroll
-        for (int i = 0; i < ITEMS; ++i) {
-            const uint32_t d = item[i] >> (16 + D0_BITS);
-            unsigned peers = 0xffffffffu;
-#pragma unroll
-            for (int b = 0; b < D1_BITS; ++b) {
-                const bool bit = (d >> b) & 1u;
-                const unsigned bal = __ballot_sync(0xffffffffu, bit);
-                peers &= bit ? bal : ~bal;
-            }
-            const uint32_t base = cnt1[warp * D1 + d];
-            const unsigned rank = __popc(peers & lt_mask);
-            __syncwarp();
-            if (rank == 0) cnt1[warp * D1 + d] = base + __popc(peers);
-            __syncwarp();
-            buf[dbase1[d] + base + rank] = item[i];
+    for (int i = 0; i < ITEMS; ++i) {
+        if (tid * ITEMS + i < m) {
+            uint16_t *c = cnt1 + (item[i] >> (16 + D0_BITS)) * THREADS + tid;
+            const uint32_t pos = *c;
+            *c = (uint16_t)(pos + 1u);
+            buf[pos] = item[i];
         }
     }
 
@@ -308,7 +336,7 @@ int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool laun
     if ((reinterpret_cast<uintptr_t>(args.G) & 15u) || (cols % 4) != 0) return 1;
     for (Variant16 &v : kVariants) {
         if (v.cap < cols) continue;
-        const Layout16 L = layout16(v.cap, v.threads / 32);
+        const Layout16 L = layout16((int)cols, v.threads);
         if (L.total > (size_t)ctx->max_smem_optin) continue;
         args.rec_stride = (long long)row_record(args.m).total;
         if (!launch) return SKIM_OK;
