@@ -116,18 +116,15 @@ struct SortedItems16 {
     {
         const uint4 a = *reinterpret_cast<const uint4 *>(items + e), b = *reinterpret_cast<const uint4 *>(items + e + 4);
         const uint32_t it[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        unsigned bad = 0u;
+        unsigned bits = 0u;
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             ks[u] = (uint16_t)(it[u] >> 16);
-            float g = 0.0f;
-            if (e + u < m) {
-                g = graw[it[u] & 0xffffu];
-                if (!(g >= 0.0f) || g > 3.0e38f) bad |= 2u;
-            }
+            const float g = (e + u < m) ? graw[it[u] & 0xffffu] : 0.0f;
+            bits |= __float_as_uint(g);
             gs[u] = g;
         }
-        return bad;
+        return bits;      // not validated here
     }
     __device__ __forceinline__ uint16_t key_at(int p) const { return (uint16_t)(items[p] >> 16); }
 };
@@ -210,9 +207,12 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
 
     // ---------------------------------------------------------------- pass 0: scan, claim slots, scatter
     {
-        uint32_t loc[EPT], s = 0;
+        uint32_t loc[EPT], s = 0, occupied = 0;
 #pragma unroll
-        for (int u = 0; u < EPT; ++u) { loc[u] = C0[tid * EPT + u]; s += loc[u]; }
+        for (int u = 0; u < EPT; ++u) { loc[u] = C0[tid * EPT + u]; s += loc[u]; occupied += loc[u] ? 1u : 0u; }
+        // occupied low-digit bins: a lower bound of the number of distinct values
+        occupied = __reduce_add_sync(0xffffffffu, occupied);
+        if (lane == 0 && occupied) atomicAdd(&ps.misc[0], (int)occupied);
         uint32_t inc = s;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -318,7 +318,20 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     }
     // ---------------------------------------------------------------- row record
     const SortedItems16 src{buf, graw};
-    const int nd = write_row_record<uint16_t, THREADS>(a, src, ps);
+    int nd = ps.misc[0];                     // more than 16 occupied bins: more than 16 distinct values
+    if (nd <= 16) {
+        // few bins: count the distinct values themselves
+        __syncthreads();
+        if (tid == 0) ps.misc[0] = 0;
+        __syncthreads();
+        int dcount = 0;
+        for (int p = tid; p < m; p += THREADS) dcount += (p == 0 || src.key_at(p) != src.key_at(p - 1)) ? 1 : 0;
+        dcount = __reduce_add_sync(0xffffffffu, dcount);
+        if (lane == 0 && dcount) atomicAdd(&ps.misc[0], dcount);
+        __syncthreads();
+        nd = ps.misc[0];
+    }
+    write_row_record<uint16_t, THREADS, false>(a, src, ps, nd);
     if (nd <= 16) {
         collect_distinct<uint16_t, THREADS>(src, m, nd, ps);
         write_distinct_values(a, nd, ps.dvals);

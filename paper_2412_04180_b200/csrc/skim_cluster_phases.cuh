@@ -87,7 +87,7 @@ struct ClusterArgs {
 // Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are
 // multiples of 16 bytes; values are binary32 whatever key type sorted the row.
 //   hdr     int nd (number of distinct values) at byte 0; float dvals[16] at byte 64
-//   seg     one 32-byte entry per segment of 32 groups (256 elements): the binary64 sums of g,
+//   seg     one 32-byte entry per segment of 64 groups (512 elements): the binary64 sums of g,
 //           g*x and g*x^2 over all earlier segments; entry nseg holds the row totals
 //   groups  one 80-byte record per group of 8 sorted elements: 8 values, 8 importances, and the
 //           binary64 sums of g and g*x from the start of the group's segment to the group's first
@@ -102,6 +102,7 @@ struct RowRecord {
     int ngrp, nseg;
 };
 constexpr int SKIM_GROUP_BYTES = 80;
+constexpr int SKIM_SEG_SHIFT = 6;                   // a segment is 64 groups (512 elements)
 constexpr float SKIM_PAD_VALUE = 3.402823466e38f;   // largest finite binary32: 0 * padding stays 0
 
 __host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
@@ -110,7 +111,7 @@ __host__ __device__ inline RowRecord row_record(int m)
 {
     RowRecord R;
     R.ngrp = (m + 7) >> 3;
-    R.nseg = (R.ngrp + 31) >> 5;
+    R.nseg = (R.ngrp + (1 << SKIM_SEG_SHIFT) - 1) >> SKIM_SEG_SHIFT;
     R.gi_bytes = (size_t)sk_entries(m) * 4;
     R.p2_bytes = ((size_t)R.ngrp * 8 + 15) & ~(size_t)15;
     size_t off = 128;
@@ -132,8 +133,8 @@ __device__ __forceinline__ void copy16(void *dst, const void *src, size_t bytes)
 }
 
 // The sorted row as the record pass sees it.  A source gives the keys and importances of one group
-// of 8 sorted elements (positions e .. e+7; the caller masks positions >= m), returns status bits
-// for bad importance values it meets, and gives single keys.
+// of 8 sorted elements (positions e .. e+7; the caller masks positions >= m), returns the OR of the
+// bit patterns of those importances if it has not validated them (else 0), and gives single keys.
 // This one: keys and importance in two shared-memory arrays, padded to whole groups.
 template <typename KeyT> struct SortedArrays {
     const KeyT *skeys;
@@ -151,7 +152,7 @@ template <typename KeyT> struct SortedArrays {
 
 // Small per-block scratch of the phases below.
 struct PhaseSmem {
-    double segtot[96][3];   // sums of every segment of 32 groups (rows of up to 24 576 elements)
+    double segtot[64][3];   // sums of every segment of 64 groups (rows of up to 24 576 elements have 48)
     float tfs[32];     // scratch of collect_distinct
     float dvals[32];   // the row's distinct values when there are at most 16
     int misc[4];       // [0] distinct count, [1] slot counter
@@ -179,15 +180,17 @@ __device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, 
     __syncthreads();
 }
 
-// Writes the row record from the sorted row in shared memory (keys and importance, padded to
-// whole groups: largest key / zero importance).  One pass: a lane takes one group of 8 elements,
-// decodes it, sums g, g*x, g*x^2 in binary64 (pairwise), a warp scan turns the 32 group sums of a
-// segment into prefix sums, and the group record goes straight to global memory; segments are
-// independent, so no warp waits for another.  The same pass counts the row's distinct values.
-// Afterwards one warp turns the segment sums into the segment table.  Call with all threads;
-// ps.misc[0..1] must have been zeroed before (and synced).  Returns nd (distinct values).
-template <typename KeyT, int THREADS, typename Src>
-__device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src &src, PhaseSmem &ps)
+// Writes the row record from the sorted row (a source, see above; padded to whole groups: largest
+// key / zero importance).  One pass: a lane takes two adjacent groups of 8 elements, decodes them,
+// stores their values and importances, sums g, g*x, g*x^2 in binary64 (pairwise); one warp scan over
+// the lanes' totals turns the 64 group sums of a segment into prefix sums, which complete the
+// group records in global memory.  Segments are independent, so no warp waits for another.
+// Afterwards one warp turns the segment sums into the segment table.  Call with all threads.
+// COUNT: the pass also counts the row's distinct values (ps.misc[0..1] zeroed before, and synced)
+// and returns the count; otherwise the caller passes the count (any number above 16 stands for
+// "more than 16") in nd_known.
+template <typename KeyT, int THREADS, bool COUNT, typename Src>
+__device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src &src, PhaseSmem &ps, int nd_known)
 {
     constexpr int NW = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -199,38 +202,56 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
     int distinct = 0;
     unsigned bad = 0u;
     for (int sgm = warp; sgm < R.nseg; sgm += NW) {
-        const int q = (sgm << 5) + lane;
-        double v0 = 0.0, v1 = 0.0, v2 = 0.0;
-        float x[8];
-        float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga;
-        if (q < R.ngrp) {
-            const int e = q << 3;
-            KeyT ks[8];
-            float gs[8];
-            bad |= src.group(e, m, ks, gs);
-            ga = make_float4(gs[0], gs[1], gs[2], gs[3]);
-            gb = make_float4(gs[4], gs[5], gs[6], gs[7]);
-            KeyT prev = e > 0 ? src.key_at(e - 1) : (KeyT)0;
+        const int q0 = (sgm << SKIM_SEG_SHIFT) + 2 * lane;
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0;       // sums of the lane's first group
+        double w0 = 0.0, w1 = 0.0, w2 = 0.0;       // sums of both
+        float first[2] = {0.0f, 0.0f};
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const bool real = e + u < m;
-                x[u] = real ? KeyOps<KeyT>::to_float(ks[u]) : SKIM_PAD_VALUE;
-                distinct += (real && (e + u == 0 || ks[u] != prev)) ? 1 : 0;
-                prev = ks[u];
-            }
-            double t0[8], t1[8], t2[8];
+        for (int h = 0; h < 2; ++h) {
+            const int q = q0 + h;
+            if (q < R.ngrp) {
+                const int e = q << 3;
+                KeyT ks[8];
+                float gs[8], x[8];
+                const unsigned gbits = src.group(e, m, ks, gs);
+                KeyT prev = (COUNT && e > 0) ? src.key_at(e - 1) : (KeyT)0;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const double g = (double)gs[u], xd = (double)x[u];      // padding: g = 0, x finite
-                t0[u] = g;
-                t1[u] = g * xd;
-                t2[u] = t1[u] * xd;
+                for (int u = 0; u < 8; ++u) {
+                    const bool real = e + u < m;
+                    x[u] = real ? KeyOps<KeyT>::to_float(ks[u]) : SKIM_PAD_VALUE;
+                    if (COUNT) {
+                        distinct += (real && (e + u == 0 || ks[u] != prev)) ? 1 : 0;
+                        prev = ks[u];
+                    }
+                }
+                float4 *d = reinterpret_cast<float4 *>(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES);
+                d[0] = make_float4(x[0], x[1], x[2], x[3]);
+                d[1] = make_float4(x[4], x[5], x[6], x[7]);
+                d[2] = make_float4(gs[0], gs[1], gs[2], gs[3]);
+                d[3] = make_float4(gs[4], gs[5], gs[6], gs[7]);
+                first[h] = x[0];
+                double t0[8], t1[8], t2[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const double g = (double)gs[u], xd = (double)x[u];      // padding: g = 0, x finite
+                    t0[u] = g;
+                    t1[u] = g * xd;
+                    t2[u] = t1[u] * xd;
+                }
+                const double v0 = ((t0[0] + t0[1]) + (t0[2] + t0[3])) + ((t0[4] + t0[5]) + (t0[6] + t0[7]));
+                const double v1 = ((t1[0] + t1[1]) + (t1[2] + t1[3])) + ((t1[4] + t1[5]) + (t1[6] + t1[7]));
+                const double v2 = ((t2[0] + t2[1]) + (t2[2] + t2[3])) + ((t2[4] + t2[5]) + (t2[6] + t2[7]));
+                // importance the source has not validated: a sign bit or a non-finite sum asks for a closer look
+                if ((gbits >> 31) || !(v0 < 1.0e300)) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (!(gs[u] >= 0.0f) || gs[u] > 3.0e38f) bad |= 2u;
+                }
+                if (h == 0) { a0 = v0; a1 = v1; a2 = v2; }
+                w0 += v0; w1 += v1; w2 += v2;
             }
-            v0 = ((t0[0] + t0[1]) + (t0[2] + t0[3])) + ((t0[4] + t0[5]) + (t0[6] + t0[7]));
-            v1 = ((t1[0] + t1[1]) + (t1[2] + t1[3])) + ((t1[4] + t1[5]) + (t1[6] + t1[7]));
-            v2 = ((t2[0] + t2[1]) + (t2[2] + t2[3])) + ((t2[4] + t2[5]) + (t2[6] + t2[7]));
         }
-        double i0 = v0, i1 = v1, i2 = v2;
+        double i0 = w0, i1 = w1, i2 = w2;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const double u0 = __shfl_up_sync(0xffffffffu, i0, off);
@@ -239,27 +260,30 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
             if (lane >= off) { i0 += u0; i1 += u1; i2 += u2; }
         }
         if (lane == 31) { ps.segtot[sgm][0] = i0; ps.segtot[sgm][1] = i1; ps.segtot[sgm][2] = i2; }
-        if (q < R.ngrp) {
-            unsigned char *gr = rec + R.groups + (size_t)q * SKIM_GROUP_BYTES;
-            float4 *d = reinterpret_cast<float4 *>(gr);
-            d[0] = make_float4(x[0], x[1], x[2], x[3]);
-            d[1] = make_float4(x[4], x[5], x[6], x[7]);
-            d[2] = ga;
-            d[3] = gb;
-            *reinterpret_cast<double2 *>(gr + 64) = make_double2(i0 - v0, i1 - v1);
-            p2[q] = i2 - v2;
-            gi[q] = x[0];
+        double e0 = i0 - w0, e1 = i1 - w1, e2 = i2 - w2;     // sums from the segment start to the lane's first group
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int q = q0 + h;
+            if (q < R.ngrp) {
+                *reinterpret_cast<double2 *>(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES + 64) = make_double2(e0, e1);
+                p2[q] = e2;
+                gi[q] = first[h];
+            }
+            e0 += a0; e1 += a1; e2 += a2;
         }
     }
-#pragma unroll
-    for (int off = 16; off; off >>= 1) distinct += __shfl_xor_sync(0xffffffffu, distinct, off);
-    if (lane == 0 && distinct) atomicAdd(&ps.misc[0], distinct);
     if (bad) atomicOr(a.status, (unsigned long long)bad);
     for (int q = R.ngrp + threadIdx.x; q < sk_entries(m); q += THREADS) gi[q] = SKIM_PAD_VALUE;
+    int nd = nd_known;
+    if (COUNT) {
+#pragma unroll
+        for (int off = 16; off; off >>= 1) distinct += __shfl_xor_sync(0xffffffffu, distinct, off);
+        if (lane == 0 && distinct) atomicAdd(&ps.misc[0], distinct);
+    }
     __syncthreads();
-    const int nd = ps.misc[0];
+    if (COUNT) nd = ps.misc[0];
     if (warp == 0) {
-        // segment table: sums over all earlier segments (4 entries per lane cover the 97 possible)
+        // segment table: sums over all earlier segments (4 entries per lane cover the 49 possible)
         double run0 = 0.0, run1 = 0.0, run2 = 0.0, loc[4][3];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {

@@ -186,11 +186,11 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
         double P0 = 0.0, P1 = 0.0, Pc = 0.0;
         if (normal) {
             if (searches) {
-                const double2 sb = __ldg(reinterpret_cast<const double2 *>(seg + (grp_i >> 5)));   // sums of the earlier segments
+                const double2 sb = __ldg(reinterpret_cast<const double2 *>(seg + (grp_i >> SKIM_SEG_SHIFT)));   // sums of the earlier segments
                 P0 = sb.x + grp.p.x;
                 P1 = sb.y + grp.p.y;
                 if (final) {
-                    Pc = __ldg(&seg[grp_i >> 5].z) + __ldg(P2 + grp_i);
+                    Pc = __ldg(&seg[grp_i >> SKIM_SEG_SHIFT].z) + __ldg(P2 + grp_i);
                     add_group<true>(grp, cntk, P0, P1, Pc);
                 } else {
                     add_group<false>(grp, cntk, P0, P1, Pc);
