@@ -14,6 +14,8 @@
  *   - greedy bit allocation                               -- Section 4.2, Algorithm 1.
  *   - scaling vector  Wq = Quant(W * alpha^-1) * alpha    -- Section 4.3, Algorithm 2.
  *   - packing rows grouped by bit-width                   -- Section 4.2, last paragraph.
+ *   - unpacking: dequantised weights and the matrix-vector product from the packed form
+ *                                                         -- Section 4 overview, Sections 4.2, 4.3.
  *
  * Readings where the paper is silent (kept identical on the CUDA side):
  *   - init: centroid j of k = sorted_row[ floor((2j+1) m / (2k)) ] (index quantiles).
@@ -394,6 +396,87 @@ int skim_oracle_emit(const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, 
                 float cv = centroids[(size_t)i * sumk + off + (j < k ? j : k - 1)];
                 lut[(size_t)i * kmax + j] = float_to_half_bits(cv);
             }
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ unpacking: dequantised weights */
+
+/* Code of element j in a packed row of `width`-bit codes (little-endian bit stream). */
+static uint32_t packed_code(const uint32_t *row_words, int64_t j, int width)
+{
+    uint32_t code = 0;
+    int64_t bit = j * width;
+    for (int t = 0; t < width; ++t) code |= ((row_words[(bit + t) / 32] >> ((bit + t) % 32)) & 1u) << t;
+    return code;
+}
+
+/*
+ * Dequantised weights from the packed form (Section 4 overview: the weights are recovered
+ * from labels, centroids and the scaling vector; Section 4.3: Wq = Quant(W * alpha^-1) * alpha;
+ * Section 4.2, last paragraph: rows are unpacked group by group).
+ *   Wq[i][j] = binary16( float(lut[i][code_ij]) * s_j )   product in binary32, then one more
+ *   round-to-nearest-even to binary16; with no scale (s == NULL) Wq is the codebook entry itself.
+ * out: [rows][cols] binary16 bit patterns, in source-row order.
+ */
+int skim_oracle_dequantize(const uint32_t *packed, const int32_t *row_order, const int64_t *group_start,
+                           const int64_t *group_word, const uint16_t *lut, const float *s, int64_t rows,
+                           int64_t cols, const int *bit_set, int n_bits, uint16_t *out)
+{
+    if (!packed || !row_order || !group_start || !group_word || !lut || !out || rows <= 0 || cols <= 0) return -1;
+    if (check_bit_set(bit_set, n_bits)) return -1;
+    int kmax = 1 << bit_set[n_bits - 1];
+    for (int b = 0; b < n_bits; ++b) {
+        int width = bit_set[b];
+        int64_t stride = skim_oracle_row_stride_words(cols, width);
+        for (int64_t p = group_start[b]; p < group_start[b + 1]; ++p) {
+            int64_t i = row_order[p];
+            const uint32_t *src = packed + group_word[b] + (p - group_start[b]) * stride;
+            for (int64_t j = 0; j < cols; ++j) {
+                uint16_t entry = lut[(size_t)i * kmax + packed_code(src, j, width)];
+                if (s) {
+                    volatile float prod = half_bits_to_float(entry) * s[j];   /* binary32 product */
+                    out[(size_t)i * cols + j] = float_to_half_bits(prod);
+                } else {
+                    out[(size_t)i * cols + j] = entry;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/*
+ * Matrix-vector product with the quantised matrix taken straight from its packed form (the
+ * inference-side consumer of the packing of Section 4.2):
+ *   y_i = sum_j float(lut[i][code_ij]) * z_j,   z_j = float(x_j) * s_j in binary32 (z = x when
+ *   s == NULL), the sum in binary64.  abs_sum (may be NULL) receives sum_j |term|, the scale of
+ *   the rounding error of a lower-precision accumulation.
+ *   x: [cols] binary16 bit patterns;  y, abs_sum: [rows] double, source-row order.
+ */
+int skim_oracle_matvec(const uint32_t *packed, const int32_t *row_order, const int64_t *group_start,
+                       const int64_t *group_word, const uint16_t *lut, const float *s, const uint16_t *x,
+                       int64_t rows, int64_t cols, const int *bit_set, int n_bits, double *y, double *abs_sum)
+{
+    if (!packed || !row_order || !group_start || !group_word || !lut || !x || !y || rows <= 0 || cols <= 0) return -1;
+    if (check_bit_set(bit_set, n_bits)) return -1;
+    int kmax = 1 << bit_set[n_bits - 1];
+    for (int b = 0; b < n_bits; ++b) {
+        int width = bit_set[b];
+        int64_t stride = skim_oracle_row_stride_words(cols, width);
+        for (int64_t p = group_start[b]; p < group_start[b + 1]; ++p) {
+            int64_t i = row_order[p];
+            const uint32_t *src = packed + group_word[b] + (p - group_start[b]) * stride;
+            double acc = 0.0, mag = 0.0;
+            for (int64_t j = 0; j < cols; ++j) {
+                volatile float z = s ? half_bits_to_float(x[j]) * s[j] : half_bits_to_float(x[j]);
+                double term = (double)half_bits_to_float(lut[(size_t)i * kmax + packed_code(src, j, width)]) * (double)z;
+                acc += term;
+                mag += fabs(term);
+            }
+            y[i] = acc;
+            if (abs_sum) abs_sum[i] = mag;
         }
     }
     return 0;

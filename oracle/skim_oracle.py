@@ -151,6 +151,47 @@ def emit(W, bits, centroids, bit_set, s=None):
                 group_word=group_word, lut=lut, codes=codes)
 
 
+def _packed_args(em, bit_set):
+    bs, _ = _bit_array(bit_set)
+    packed = np.ascontiguousarray(em["packed"], dtype=np.uint32)
+    if packed.size == 0:
+        packed = np.zeros(4, dtype=np.uint32)
+    return (bs, packed, np.ascontiguousarray(em["row_order"], dtype=np.int32),
+            np.ascontiguousarray(em["group_start"], dtype=np.int64), np.ascontiguousarray(em["group_word"], dtype=np.int64),
+            np.ascontiguousarray(em["lut"], dtype=np.uint16))
+
+
+def dequantize(em, cols, bit_set, s=None):
+    """Dequantised weights (float16 [rows, cols]) from an emit() result."""
+    bs, packed, row_order, gs, gw, lut = _packed_args(em, bit_set)
+    rows = lut.shape[0]
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+    out = np.zeros((rows, cols), dtype=np.uint16)
+    rc = lib().skim_oracle_dequantize(_p(packed), _p(row_order), _p(gs), _p(gw), _p(lut), _p(s), C.c_int64(rows),
+                                      C.c_int64(cols), _p(bs), C.c_int(len(bs)), _p(out))
+    if rc:
+        raise ValueError(f"skim_oracle_dequantize failed ({rc})")
+    return out.view(np.float16)
+
+
+def matvec(em, cols, bit_set, x, s=None):
+    """y = Wq x from the packed form; returns (y float64 [rows], sum of |terms| float64 [rows])."""
+    bs, packed, row_order, gs, gw, lut = _packed_args(em, bit_set)
+    rows = lut.shape[0]
+    x = np.ascontiguousarray(x)
+    assert x.dtype == np.float16 and x.shape == (cols,)
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+    y = np.zeros(rows, dtype=np.float64)
+    mag = np.zeros(rows, dtype=np.float64)
+    rc = lib().skim_oracle_matvec(_p(packed), _p(row_order), _p(gs), _p(gw), _p(lut), _p(s), _p(x.view(np.uint16)),
+                                  C.c_int64(rows), C.c_int64(cols), _p(bs), C.c_int(len(bs)), _p(y), _p(mag))
+    if rc:
+        raise ValueError(f"skim_oracle_matvec failed ({rc})")
+    return y, mag
+
+
 def scale_loss_grad(W, importance, labels, alpha, want_grad=True):
     W = np.ascontiguousarray(W)
     assert W.dtype == np.float16
