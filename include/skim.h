@@ -12,6 +12,8 @@
  *   skim_quantize         labels at the allocated width, packed by width group, and the
  *                         per-row codebook                      (Algorithm 3, second loop;
  *                                                                Section 4.2, last paragraph)
+ *   skim_dequantize       the fp16 matrix back from packed codes, codebooks and alpha
+ *   skim_matvec           y = Wq x from the packed form   (Section 4.2, last paragraph; 4.3)
  *   skim_apply_scale      installs the scaling vector alpha: all later calls cluster
  *                         W * alpha^-1                          (Section 4.3, Algorithm 2)
  *   skim_cluster_rows_at  re-clustering at the already allocated widths inside the
@@ -178,6 +180,35 @@ int skim_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, 
 int skim_quantize_static(void *cuda_stream, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
                          const uint8_t *bits, const float *centroids, const int *bit_set, int n_bits,
                          uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);
+
+/*
+ * Unpacking (Section 4.2, last paragraph: rows of equal width are stored together and unpacked
+ * group by group; Section 4 overview and Section 4.3: the dequantised weight is the codebook
+ * entry of its label times the scaling vector, Wq = Quant(W * alpha^-1) * alpha).
+ * Inputs are the outputs of skim_quantize: packed, row_order [rows], group_info [2*(n_bits+1)],
+ * lut [rows][2^b_max] (indexed by SOURCE row), all device pointers; s (device, [cols], may be
+ * NULL for alpha = 1) is the scaling vector itself, not its reciprocal.  No workspace is used.
+ *   out  [rows][ld_out] binary16, source-row order:
+ *        out[i][j] = binary16( float(lut[i][code_ij]) * s_j ), the product taken in binary32 and
+ *        rounded to nearest even once more; with s == NULL the codebook entry itself.
+ * Rows that skim_quantize skipped (width outside bit_set) are left untouched.
+ * cols is limited by shared memory (the per-column vector of a block sits there: about 58 000 on
+ * B200); ld_out >= cols.
+ */
+int skim_dequantize(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order, const int64_t *group_info,
+                    const uint16_t *lut, const float *s, int64_t rows, int64_t cols, const int *bit_set,
+                    int n_bits, uint16_t *out, int64_t ld_out);
+
+/*
+ * y = Wq x straight from the packed form, Wq as defined for skim_dequantize but never rounded to
+ * binary16 or stored: y_i = sum_j float(lut[i][code_ij]) * z_j with z_j = float(x_j) * s_j in
+ * binary32 (z = x when s == NULL).  The sum is accumulated in binary32 (per lane in element
+ * order, then a 5-level tree), so |y_i - exact| <= (cols/32 + 8) * 2^-24 * sum_j |term_ij|.
+ *   x  [cols] binary16 bit patterns (device);  y  out [rows] binary32, source-row order (device)
+ */
+int skim_matvec(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order, const int64_t *group_info,
+                const uint16_t *lut, const float *s, const uint16_t *x, int64_t rows, int64_t cols,
+                const int *bit_set, int n_bits, float *y);
 
 /*
  * Algorithm 2, inner repeat: `steps` Adam updates (Section 5.1: learning rate lr0, multiplied

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libskim.so")
-SOURCES = ["skim_api.cu", "skim_cluster.cu", "skim_cluster16.cu", "skim_lloyd.cu", "skim_allocate.cu", "skim_quantize.cu", "skim_scale.cu"]
+SOURCES = ["skim_api.cu", "skim_cluster.cu", "skim_cluster16.cu", "skim_lloyd.cu", "skim_allocate.cu", "skim_quantize.cu", "skim_unpack.cu", "skim_scale.cu"]
 
 
 def _stale() -> bool:

@@ -237,6 +237,47 @@ int skim_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, 
     return skim_launch_quantize(ctx, W, rows, cols, ld, bits, centroids, bs, packed, row_order, group_info, lut);
 }
 
+namespace {
+int check_unpack(const skim_ctx *ctx, int64_t rows, int64_t cols)
+{
+    if (rows < 0 || rows > 0x7fffffff || cols < 1 || cols > 0x7fffff00) return SKIM_ERR_SHAPE;
+    // the per-column vector of one block lives in shared memory
+    if ((size_t)((cols + 255) / 256 * 256) * sizeof(float) > (size_t)ctx->max_smem_optin) return SKIM_ERR_SHAPE;
+    return SKIM_OK;
+}
+}  // namespace
+
+int skim_dequantize(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order, const int64_t *group_info,
+                    const uint16_t *lut, const float *s, int64_t rows, int64_t cols, const int *bit_set, int n_bits,
+                    uint16_t *out, int64_t ld_out)
+{
+    if (!ctx || !packed || !row_order || !group_info || !lut || !out) return SKIM_ERR_NULL;
+    SkimBits bs;
+    int rc = skim_check_bits(bit_set, n_bits, &bs);
+    if (rc) return rc;
+    rc = check_unpack(ctx, rows, cols);
+    if (rc) return rc;
+    if (ld_out < cols) return SKIM_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_dequantize(ctx, packed, row_order, group_info, lut, s, rows, cols, bs, out, ld_out);
+}
+
+int skim_matvec(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order, const int64_t *group_info,
+                const uint16_t *lut, const float *s, const uint16_t *x, int64_t rows, int64_t cols,
+                const int *bit_set, int n_bits, float *y)
+{
+    if (!ctx || !packed || !row_order || !group_info || !lut || !x || !y) return SKIM_ERR_NULL;
+    SkimBits bs;
+    int rc = skim_check_bits(bit_set, n_bits, &bs);
+    if (rc) return rc;
+    rc = check_unpack(ctx, rows, cols);
+    if (rc) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_matvec(ctx, packed, row_order, group_info, lut, s, x, rows, cols, bs, y);
+}
+
 int skim_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
                       int64_t ld, const uint8_t *labels, float *alpha, int steps, float lr0, float decay,
                       int decay_every, double *loss_trace)

@@ -113,6 +113,12 @@ int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const Sk
 int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
                          const uint8_t *bits, const float *centroids, const SkimBits &bs,
                          uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);
+int skim_launch_dequantize(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order, const int64_t *group_info,
+                           const uint16_t *lut, const float *s, int64_t rows, int64_t cols, const SkimBits &bs,
+                           uint16_t *out, int64_t ld_out);
+int skim_launch_matvec(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order, const int64_t *group_info,
+                       const uint16_t *lut, const float *s, const uint16_t *x, int64_t rows, int64_t cols,
+                       const SkimBits &bs, float *y);
 int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
                              int64_t cols, int64_t ld, const uint8_t *labels, float *alpha, int steps,
                              float lr0, float decay, int decay_every, double *loss_trace);

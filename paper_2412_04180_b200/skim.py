@@ -21,7 +21,7 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
            "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits",
-           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_scale_update", "skim_host_staging_bytes",
+           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
            "skim_kernel_times", "skim_strerror"]
 
@@ -206,6 +206,33 @@ class Skim:
         _chk(lib().skim_quantize(self._h, _ptr(W), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols), _ptr(bits),
                                  _ptr(centroids), arr, C.c_int(nb), _ptr(out["packed"]), _ptr(out["row_order"]),
                                  _ptr(out["group_info"]), _ptr(out["lut"])), "skim_quantize")
+        return out
+
+    def dequantize(self, q, cols, bit_set, s=None, out=None):
+        """float16 [rows, cols] dequantised weights from a quantize() result ``q``; ``s`` is the scaling vector."""
+        rows = q["row_order"].numel()
+        arr, nb, _ = _bits(bit_set)
+        if s is not None:
+            _dev(s, torch.float32, "s")
+        if out is None:
+            out = torch.empty((rows, cols), dtype=torch.float16, device=q["packed"].device)
+        _chk(lib().skim_dequantize(self._h, _ptr(q["packed"]), _ptr(q["row_order"]), _ptr(q["group_info"]),
+                                   _ptr(q["lut"]), _ptr(s), C.c_int64(rows), C.c_int64(cols), arr, C.c_int(nb),
+                                   _ptr(out), C.c_int64(out.stride(0))), "skim_dequantize")
+        return out
+
+    def matvec(self, q, cols, bit_set, x, s=None, out=None):
+        """float32 [rows] = Wq x from a quantize() result ``q`` and a float16 vector ``x`` [cols]."""
+        rows = q["row_order"].numel()
+        arr, nb, _ = _bits(bit_set)
+        _dev(x, torch.float16, "x")
+        if s is not None:
+            _dev(s, torch.float32, "s")
+        if out is None:
+            out = torch.empty((rows,), dtype=torch.float32, device=x.device)
+        _chk(lib().skim_matvec(self._h, _ptr(q["packed"]), _ptr(q["row_order"]), _ptr(q["group_info"]), _ptr(q["lut"]),
+                               _ptr(s), _ptr(x), C.c_int64(rows), C.c_int64(cols), arr, C.c_int(nb), _ptr(out)),
+             "skim_matvec")
         return out
 
     def scale_update(self, W, importance, labels, alpha, steps=120, lr0=0.01, decay=0.5, decay_every=40,
