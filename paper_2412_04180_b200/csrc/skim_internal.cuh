@@ -45,9 +45,11 @@ struct SkimWorkspace {
     double *alpha64;             // [cols]     scale-update master copy of alpha
     double *adam_m;              // [cols]
     double *adam_v;              // [cols]
-    double *ralpha;              // [cols]     1 / alpha (binary64)
-    double *loss_part;           // [SKIM_SCALE_MAX_CTAS]
-    double *grad_part;           // [SKIM_SCALE_MAX_CTAS][cols]
+    double *ralpha;              // [cols]     (unused)
+    double *loss_part;           // [rows]     scale update: loss of every row
+    double *grad_part;           // [SKIM_SCALE_MAX_CTAS][cols]  partial gradients of the row ranges
+    double *scale_const;         // [rows][16][2]  scale update: per-cluster constants (sum g, sum g w^2)
+    double *scale_cq;            // [rows][16][2]  scale update: per-cluster centroid and gradient factor
     unsigned char *cluster_scratch;  // [min(rows, SKIM_CLUSTER_CHUNK_ROWS)] row records of the clustering
     size_t bytes;
 };
@@ -78,8 +80,10 @@ static inline SkimWorkspace skim_carve(void *base, int64_t rows, int64_t cols)
     w.adam_m = (double *)take((size_t)cols * 8);
     w.adam_v = (double *)take((size_t)cols * 8);
     w.ralpha = (double *)take((size_t)cols * 8);
-    w.loss_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * 8);
+    w.loss_part = (double *)take((size_t)(rows > SKIM_SCALE_MAX_CTAS ? rows : SKIM_SCALE_MAX_CTAS) * 8);
     w.grad_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * (size_t)cols * 8);
+    w.scale_const = (double *)take((size_t)rows * 16 * 2 * 8);
+    w.scale_cq = (double *)take((size_t)rows * 16 * 2 * 8);
     w.cluster_scratch = (unsigned char *)take((size_t)(rows < SKIM_CLUSTER_CHUNK_ROWS ? rows : SKIM_CLUSTER_CHUNK_ROWS) *
                                               skim_cluster_record_bytes(cols));
     w.bytes = off;

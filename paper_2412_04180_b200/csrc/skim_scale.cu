@@ -4,148 +4,236 @@
 //   loss(alpha) = sum_ij g_ij (W_ij - alpha_j c_{i,l_ij})^2,
 //   c_ik        = sum_{j in k} g_ij W_ij / alpha_j  /  sum_{j in k} g_ij   (re-fitted each step)
 //
-// Per Adam step two kernels run:
-//   skim_scale_rows_kernel  a fixed set of blocks, each walking a contiguous chunk of rows.  For
-//       a row it makes three passes over (W, g, label): cluster sums -> centroids; residual
-//       sums; gradient terms, which it adds to a per-block column accumulator in shared memory.
-//       The first pass comes from HBM, the other two hit L2.  Per-thread private accumulator
-//       slots in shared memory keep every sum in binary64 without atomics.
-//   skim_scale_adam_kernel  sums the per-block column partials in block order (deterministic),
-//       applies the Adam update to the binary64 master copy of alpha and refreshes 1/alpha.
+// Per Adam step the matrix is read twice, by two kernels:
+//   skim_scale_sums_kernel  one warp per row.  Per cluster k of the row it forms, in binary64,
+//       S_k = sum g w / alpha,  A_k = sum g w alpha,  B_k = sum g alpha^2  (sums over the members).
+//       With the per-call constants G_k = sum g and D_k = sum g w^2 (the same kernel, run once in
+//       its INIT form) these give the centroid c_k = S_k / G_k, the row's loss
+//       sum_k D_k - 2 c_k A_k + c_k^2 B_k, and the factor q_k = 2 (A_k - c_k B_k) / G_k through which the
+//       re-fitted centroid enters the gradient -- without a second pass over the row.  A lane adds
+//       its elements into accumulator slots of its own in shared memory (one per cluster and
+//       sum), so no atomics are needed and every sum has a fixed order.
+//   skim_scale_grad_kernel  a thread owns four columns and walks a range of rows:
+//       d loss / d alpha_j = sum_i  -2 g c (w - alpha_j c) + q g w / alpha_j^2   (c, q of the element's
+//       cluster, read from the 512-byte table the first kernel left for the row), accumulated in
+//       registers; the row ranges leave partial gradients that the Adam kernel adds in a fixed order.
+//   skim_scale_adam_kernel  sums the partials and the rows' losses (deterministic), applies the
+//       Adam update to the binary64 master copy of alpha.
 #include "skim_internal.cuh"
 
 namespace {
 
-constexpr int KC = 16;  // clusters per row at most (4 bits)
+constexpr int KC = 16;      // clusters per row at most (4 bits)
+constexpr int SW = 4;       // warps (rows) per block of the sums kernel
+constexpr int NSUM = 3;
+constexpr int GT = 256;     // threads of a gradient block
+constexpr int GC = 4;       // columns per thread
 
 struct ScaleArgs {
     const uint16_t *W;
     const float *G;
     const uint8_t *labels;
     const double *alpha;
-    const double *ralpha;
     int64_t rows, ld;
     int cols;
-    int rows_per_block;
-    double *grad_part;   // [gridDim.x][cols]
-    double *loss_part;   // [gridDim.x]
+    int vec;                // rows of W, G and labels allow the vector loads of both kernels
+    double2 *tconst;        // [rows][KC]  (G_k, D_k)
+    double2 *tq;            // [rows][KC]  (c_k, q_k)
+    double *loss_row;       // [rows]
+    double *grad_part;      // [row ranges][cols]
+    int rows_per_range;
 };
 
-template <int THREADS>
-__global__ void __launch_bounds__(THREADS) skim_scale_rows_kernel(ScaleArgs a)
+// Eight consecutive elements of a row starting at e0 (a multiple of 8); entries at or beyond cols come
+// back with zero importance, label 0 and alpha 1.
+template <bool VEC>
+__device__ __forceinline__ void load8(const ScaleArgs &a, int64_t row, int e0, float *w, float *g, int *l, double *al)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *colacc = reinterpret_cast<double *>(smem_raw);            // [cols]
-    double *acc0 = colacc + a.cols;                                   // [KC][THREADS]
-    double *acc1 = acc0 + KC * THREADS;                               // [KC][THREADS]
-    double *Gv = acc1 + KC * THREADS;                                 // [KC]
-    double *Cv = Gv + KC;                                             // [KC]
-    double *Rv = Cv + KC;                                             // [KC]
-    double *red = Rv + KC;                                            // [32]
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int NW = THREADS / 32;
-
-    for (int e = tid; e < a.cols; e += THREADS) colacc[e] = 0.0;
-    double loss = 0.0;
-    const int64_t r0 = (int64_t)blockIdx.x * a.rows_per_block;
-    const int64_t r1 = min(a.rows, r0 + a.rows_per_block);
-    for (int64_t row = r0; row < r1; ++row) {
-        const uint16_t *Wr = a.W + row * a.ld;
-        const float *Gr = a.G + row * a.ld;
-        const uint8_t *Lr = a.labels + row * (int64_t)a.cols;
+    const uint16_t *Wr = a.W + row * a.ld;
+    const float *Gr = a.G + row * a.ld;
+    const uint8_t *Lr = a.labels + row * (int64_t)a.cols;
+    if (VEC && e0 + 8 <= a.cols) {
+        const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(Wr + e0));
+        const float4 ga = __ldg(reinterpret_cast<const float4 *>(Gr + e0)), gb = __ldg(reinterpret_cast<const float4 *>(Gr + e0 + 4));
+        const uint2 lv = __ldg(reinterpret_cast<const uint2 *>(Lr + e0));
+        const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+        const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
 #pragma unroll
-        for (int k = 0; k < KC; ++k) { acc0[k * THREADS + tid] = 0.0; acc1[k * THREADS + tid] = 0.0; }
-        // pass 1: G_k = sum g, S_k = sum g w / alpha
-        for (int e = tid; e < a.cols; e += THREADS) {
-            const int l = Lr[e] & (KC - 1);
-            const double g = (double)Gr[e];
-            const double w = (double)__half2float(__ushort_as_half(Wr[e]));
-            acc0[l * THREADS + tid] += g;
-            acc1[l * THREADS + tid] += g * w * a.ralpha[e];
+        for (int u = 0; u < 8; ++u) {
+            w[u] = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+            g[u] = gg[u];
+            l[u] = (int)(((u < 4 ? lv.x : lv.y) >> (8 * (u & 3))) & (KC - 1));
         }
-        __syncthreads();
-        for (int k = warp; k < KC; k += NW) {
-            double s0 = 0.0, s1 = 0.0;
-            for (int t = lane; t < THREADS; t += 32) { s0 += acc0[k * THREADS + t]; s1 += acc1[k * THREADS + t]; }
 #pragma unroll
-            for (int off = 16; off; off >>= 1) {
-                s0 += __shfl_xor_sync(0xffffffffu, s0, off);
-                s1 += __shfl_xor_sync(0xffffffffu, s1, off);
-            }
-            if (lane == 0) { Gv[k] = s0; Cv[k] = s0 > 0.0 ? s1 / s0 : 0.0; }
+        for (int u = 0; u < 8; u += 2) {
+            const double2 av = __ldg(reinterpret_cast<const double2 *>(a.alpha + e0 + u));
+            al[u] = av.x; al[u + 1] = av.y;
         }
-        __syncthreads();
+    } else {
 #pragma unroll
-        for (int k = 0; k < KC; ++k) acc0[k * THREADS + tid] = 0.0;
-        // pass 2: residuals r = w - alpha c; loss; R_k = sum g r alpha
-        for (int e = tid; e < a.cols; e += THREADS) {
-            const int l = Lr[e] & (KC - 1);
-            const double g = (double)Gr[e];
-            const double w = (double)__half2float(__ushort_as_half(Wr[e]));
-            const double al = a.alpha[e];
-            const double r = w - al * Cv[l];
-            loss = fma(g * r, r, loss);
-            acc0[l * THREADS + tid] += g * r * al;
+        for (int u = 0; u < 8; ++u) {
+            const bool in = e0 + u < a.cols;
+            w[u] = in ? __half2float(__ushort_as_half(Wr[e0 + u])) : 0.0f;
+            g[u] = in ? Gr[e0 + u] : 0.0f;
+            l[u] = in ? (int)(Lr[e0 + u] & (KC - 1)) : 0;
+            al[u] = in ? a.alpha[e0 + u] : 1.0;
         }
-        __syncthreads();
-        for (int k = warp; k < KC; k += NW) {
-            double s0 = 0.0;
-            for (int t = lane; t < THREADS; t += 32) s0 += acc0[k * THREADS + t];
-#pragma unroll
-            for (int off = 16; off; off >>= 1) s0 += __shfl_xor_sync(0xffffffffu, s0, off);
-            if (lane == 0) Rv[k] = s0;
-        }
-        __syncthreads();
-        // pass 3: d loss / d alpha_j, both terms (directly, and through the re-fitted centroid)
-        for (int e = tid; e < a.cols; e += THREADS) {
-            const int l = Lr[e] & (KC - 1);
-            const double g = (double)Gr[e];
-            const double w = (double)__half2float(__ushort_as_half(Wr[e]));
-            const double al = a.alpha[e], ra = a.ralpha[e];
-            const double c = Cv[l];
-            const double r = w - al * c;
-            double d = -2.0 * g * r * c;
-            if (Gv[l] > 0.0) d += 2.0 * Rv[l] * g * w * ra * ra / Gv[l];
-            colacc[e] += d;
-        }
-        __syncthreads();
-    }
-    for (int e = tid; e < a.cols; e += THREADS) a.grad_part[(int64_t)blockIdx.x * a.cols + e] = colacc[e];
-#pragma unroll
-    for (int off = 16; off; off >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, off);
-    if (lane == 0) red[warp] = loss;
-    __syncthreads();
-    if (tid == 0) {
-        double s = 0.0;
-        for (int w = 0; w < NW; ++w) s += red[w];
-        a.loss_part[blockIdx.x] = s;
     }
 }
 
-__global__ void skim_scale_adam_kernel(const double *__restrict__ grad_part, const double *__restrict__ loss_part,
-                                       int nblocks, int cols, double *alpha, double *ralpha, double *m1, double *m2,
-                                       double lr, double beta1, double beta2, double bc1, double bc2, double eps,
-                                       double *loss_out)
+// INIT: the per-call constants (G_k, D_k) of every row.  Otherwise: (c_k, q_k) and the row's loss.
+template <bool INIT, bool VEC>
+__global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
 {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j == 0 && loss_out) {
-        double s = 0.0;
-        for (int b = 0; b < nblocks; ++b) s += loss_part[b];
-        *loss_out = s;
+    extern __shared__ __align__(16) double slots_all[];       // [SW][NSUM * KC][32]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * SW + warp;
+    if (row >= a.rows) return;
+    double *slot = slots_all + (size_t)warp * (NSUM * KC * 32) + lane;   // entry (s, k) at slot[(s * KC + k) * 32]
+#pragma unroll
+    for (int q = 0; q < NSUM * KC; ++q) slot[q * 32] = 0.0;
+    for (int e0 = lane * 8; e0 < a.cols; e0 += 256) {
+        float w[8], g[8];
+        int l[8];
+        double al[8];
+        load8<VEC>(a, row, e0, w, g, l, al);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const double gd = (double)g[u], wd = (double)w[u];
+            const double gw = gd * wd;
+            double *sl = slot + l[u] * 32;
+            if (INIT) {
+                sl[0] += gd;
+                sl[KC * 32] += gw * wd;
+            } else {
+                sl[0] += gw * __drcp_rn(al[u]);
+                sl[KC * 32] += gw * al[u];
+                sl[2 * KC * 32] += gd * al[u] * al[u];
+            }
+        }
     }
+    __syncwarp();
+    // lane L adds up entry L (and L + 32) over the 32 lanes' slots, starting at its own (no bank conflicts)
+    const double *base = slots_all + (size_t)warp * (NSUM * KC * 32);
+    double v0 = 0.0, v1 = 0.0;
+    for (int t = 0; t < 32; ++t) {
+        const int src = (t + lane) & 31;
+        v0 += base[lane * 32 + src];
+        if (lane < NSUM * KC - 32) v1 += base[(lane + 32) * 32 + src];
+    }
+    // sums 0 and 1 of cluster k sit in lanes k and 16 + k (v0), sum 2 in lane k (v1)
+    const double s0 = v0, s1 = __shfl_sync(0xffffffffu, v0, (lane & 15) + 16), s2 = v1;
+    double loss_k = 0.0;
+    if (lane < KC) {
+        if (INIT) {
+            a.tconst[row * KC + lane] = make_double2(s0, s1);
+        } else {
+            const double2 gdk = a.tconst[row * KC + lane];
+            double c = 0.0, q = 0.0;
+            if (gdk.x > 0.0) {
+                c = s0 / gdk.x;
+                q = 2.0 * (s1 - c * s2) / gdk.x;
+                loss_k = gdk.y - 2.0 * c * s1 + c * c * s2;
+            }
+            a.tq[row * KC + lane] = make_double2(c, q);
+        }
+    }
+    if (!INIT) {
+#pragma unroll
+        for (int off = 8; off; off >>= 1) loss_k += __shfl_down_sync(0xffffffffu, loss_k, off);
+        if (lane == 0) a.loss_row[row] = loss_k;
+    }
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(GT) skim_scale_grad_kernel(ScaleArgs a)
+{
+    const int j0 = (blockIdx.x * GT + threadIdx.x) * GC;
+    const int64_t r0 = (int64_t)blockIdx.y * a.rows_per_range;
+    const int64_t r1 = min(a.rows, r0 + a.rows_per_range);
+    if (j0 >= a.cols) return;
+    double al[GC], rr[GC], acc[GC];
+#pragma unroll
+    for (int u = 0; u < GC; ++u) {
+        al[u] = j0 + u < a.cols ? a.alpha[j0 + u] : 1.0;
+        const double r = __drcp_rn(al[u]);
+        rr[u] = r * r;
+        acc[u] = 0.0;
+    }
+    const bool full = VEC && j0 + GC <= a.cols;
+#pragma unroll 2
+    for (int64_t row = r0; row < r1; ++row) {
+        const uint16_t *Wr = a.W + row * a.ld + j0;
+        const float *Gr = a.G + row * a.ld + j0;
+        const uint8_t *Lr = a.labels + row * (int64_t)a.cols + j0;
+        float w[GC], g[GC];
+        int l[GC];
+        if (full) {
+            const uint2 wv = __ldg(reinterpret_cast<const uint2 *>(Wr));
+            const float4 gv = __ldg(reinterpret_cast<const float4 *>(Gr));
+            const uint32_t lv = __ldg(reinterpret_cast<const uint32_t *>(Lr));
+            w[0] = __half2float(__ushort_as_half((uint16_t)(wv.x & 0xffffu)));
+            w[1] = __half2float(__ushort_as_half((uint16_t)(wv.x >> 16)));
+            w[2] = __half2float(__ushort_as_half((uint16_t)(wv.y & 0xffffu)));
+            w[3] = __half2float(__ushort_as_half((uint16_t)(wv.y >> 16)));
+            g[0] = gv.x; g[1] = gv.y; g[2] = gv.z; g[3] = gv.w;
+#pragma unroll
+            for (int u = 0; u < GC; ++u) l[u] = (int)((lv >> (8 * u)) & (KC - 1));
+        } else {
+#pragma unroll
+            for (int u = 0; u < GC; ++u) {
+                const bool in = j0 + u < a.cols;
+                w[u] = in ? __half2float(__ushort_as_half(Wr[u])) : 0.0f;
+                g[u] = in ? Gr[u] : 0.0f;
+                l[u] = in ? (int)(Lr[u] & (KC - 1)) : 0;
+            }
+        }
+        const double2 *tq = a.tq + row * KC;
+#pragma unroll
+        for (int u = 0; u < GC; ++u) {
+            const double2 cq = __ldg(tq + l[u]);
+            const double gd = (double)g[u], wd = (double)w[u];
+            const double res = wd - al[u] * cq.x;
+            acc[u] += gd * (cq.y * wd * rr[u] - 2.0 * cq.x * res);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < GC; ++u)
+        if (j0 + u < a.cols) a.grad_part[(int64_t)blockIdx.y * a.cols + j0 + u] = acc[u];
+}
+
+__global__ void __launch_bounds__(256) skim_scale_adam_kernel(const double *__restrict__ grad_part,
+                                                               const double *__restrict__ loss_row, int nranges,
+                                                               int64_t rows, int cols, double *alpha, double *m1,
+                                                               double *m2, double lr, double beta1, double beta2,
+                                                               double bc1, double bc2, double eps, double *loss_out)
+{
+    __shared__ double red[256];
+    if (blockIdx.x == gridDim.x - 1) {
+        // the last block adds the rows' losses: strided partial sums, then a fixed tree
+        double s = 0.0;
+        for (int64_t i = threadIdx.x; i < rows; i += 256) s += loss_row[i];
+        red[threadIdx.x] = s;
+        __syncthreads();
+        for (int off = 128; off; off >>= 1) {
+            if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0 && loss_out) *loss_out = red[0];
+        return;
+    }
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= cols) return;
     double g = 0.0;
-    for (int b = 0; b < nblocks; ++b) g += grad_part[(int64_t)b * cols + j];
+    for (int b = 0; b < nranges; ++b) g += grad_part[(int64_t)b * cols + j];
     const double a1 = beta1 * m1[j] + (1.0 - beta1) * g;
     const double a2 = beta2 * m2[j] + (1.0 - beta2) * g * g;
     m1[j] = a1;
     m2[j] = a2;
-    const double al = alpha[j] - lr * (a1 / bc1) / (sqrt(a2 / bc2) + eps);
-    alpha[j] = al;
-    ralpha[j] = 1.0 / al;
+    alpha[j] = alpha[j] - lr * (a1 / bc1) / (sqrt(a2 / bc2) + eps);
 }
 
-__global__ void skim_scale_init_kernel(const float *__restrict__ alpha32, int cols, double *alpha, double *ralpha,
+__global__ void skim_scale_init_kernel(const float *__restrict__ alpha32, int cols, double *alpha,
                                        double *m1, double *m2, unsigned long long *status)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -153,7 +241,6 @@ __global__ void skim_scale_init_kernel(const float *__restrict__ alpha32, int co
     const float v = alpha32[j];
     if (!(v > 0.0f) || v > 3.0e38f) atomicOr(status, (unsigned long long)SKIM_STATUS_BAD_SCALE);
     alpha[j] = (double)v;
-    ralpha[j] = 1.0 / (double)v;
     m1[j] = 0.0;
     m2[j] = 0.0;
 }
@@ -164,8 +251,6 @@ __global__ void skim_scale_finish_kernel(const double *__restrict__ alpha, int c
     if (j < cols) alpha32[j] = (float)alpha[j];
 }
 
-size_t scale_smem(int cols, int threads) { return ((size_t)cols + 2 * KC * (size_t)threads + 3 * KC + 32) * 8; }
-
 }  // namespace
 
 int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
@@ -173,18 +258,8 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
                              int decay_every, double *loss_trace)
 {
     SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
-    int threads = 256;
-    size_t smem = scale_smem((int)cols, threads);
-    if (smem > (size_t)ctx->max_smem_optin) { threads = 128; smem = scale_smem((int)cols, threads); }
-    if (smem > (size_t)ctx->max_smem_optin) return SKIM_ERR_SHAPE;
-    int nblocks = (int)(rows < SKIM_SCALE_MAX_CTAS ? rows : SKIM_SCALE_MAX_CTAS);
-    const int per = (int)((rows + nblocks - 1) / nblocks);
-    nblocks = (int)((rows + per - 1) / per);
-    auto kernel = threads == 256 ? skim_scale_rows_kernel<256> : skim_scale_rows_kernel<128>;
-    SKIM_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const unsigned cb = (unsigned)((cols + 255) / 256);
-    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.ralpha, ws.adam_m, ws.adam_v,
-                                                        ws.status);
+    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.adam_m, ws.adam_v, ws.status);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     ScaleArgs a;
@@ -192,27 +267,48 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
     a.G = importance;
     a.labels = labels;
     a.alpha = ws.alpha64;
-    a.ralpha = ws.ralpha;
     a.rows = rows;
     a.ld = ld;
     a.cols = (int)cols;
-    a.rows_per_block = per;
+    a.vec = ((reinterpret_cast<uintptr_t>(W) & 15u) == 0 && (reinterpret_cast<uintptr_t>(importance) & 15u) == 0 &&
+             (reinterpret_cast<uintptr_t>(labels) & 7u) == 0 && ld % 8 == 0 && cols % 8 == 0) ? 1 : 0;
+    a.tconst = reinterpret_cast<double2 *>(ws.scale_const);
+    a.tq = reinterpret_cast<double2 *>(ws.scale_cq);
+    a.loss_row = ws.loss_part;
     a.grad_part = ws.grad_part;
-    a.loss_part = ws.loss_part;
+    // gradient kernel: column tiles x row ranges, about four blocks per SM in all
+    const int tiles = (int)((cols + GT * GC - 1) / (GT * GC));
+    int ranges = (4 * ctx->sm_count + tiles - 1) / tiles;
+    if (ranges > SKIM_SCALE_MAX_CTAS) ranges = SKIM_SCALE_MAX_CTAS;
+    if (ranges > rows) ranges = (int)rows;
+    a.rows_per_range = (int)((rows + ranges - 1) / ranges);
+    ranges = (int)((rows + a.rows_per_range - 1) / a.rows_per_range);
+    const size_t smem = (size_t)SW * NSUM * KC * 32 * sizeof(double);
+    const unsigned sum_blocks = (unsigned)((rows + SW - 1) / SW);
+    auto sums_init = a.vec ? skim_scale_sums_kernel<true, true> : skim_scale_sums_kernel<true, false>;
+    auto sums_step = a.vec ? skim_scale_sums_kernel<false, true> : skim_scale_sums_kernel<false, false>;
+    auto grad = a.vec ? skim_scale_grad_kernel<true> : skim_scale_grad_kernel<false>;
+    SKIM_CUDA_OK(cudaFuncSetAttribute(sums_init, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    SKIM_CUDA_OK(cudaFuncSetAttribute(sums_step, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    sums_init<<<sum_blocks, SW * 32, smem, ctx->stream>>>(a);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
     const double beta1 = 0.9, beta2 = 0.999, eps = 1e-8;
     double p1 = 1.0, p2 = 1.0, lr = (double)lr0;
     for (int t = 0; t < steps; ++t) {
         if (t > 0 && t % decay_every == 0) lr *= (double)decay;
         p1 *= beta1;
         p2 *= beta2;
-        kernel<<<nblocks, threads, smem, ctx->stream>>>(a);
+        sums_step<<<sum_blocks, SW * 32, smem, ctx->stream>>>(a);
         SKIM_CUDA_OK(cudaGetLastError());
-        skim_scale_adam_kernel<<<cb, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, nblocks, (int)cols, ws.alpha64,
-                                                            ws.ralpha, ws.adam_m, ws.adam_v, lr, beta1, beta2,
-                                                            1.0 - p1, 1.0 - p2, eps,
-                                                            loss_trace ? loss_trace + t : nullptr);
+        grad<<<dim3((unsigned)tiles, (unsigned)ranges), GT, 0, ctx->stream>>>(a);
         SKIM_CUDA_OK(cudaGetLastError());
-        ctx->launches += 2;
+        skim_scale_adam_kernel<<<cb + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
+                                                                ws.alpha64, ws.adam_m, ws.adam_v, lr, beta1, beta2,
+                                                                1.0 - p1, 1.0 - p2, eps,
+                                                                loss_trace ? loss_trace + t : nullptr);
+        SKIM_CUDA_OK(cudaGetLastError());
+        ctx->launches += 3;
     }
     skim_scale_finish_kernel<<<cb, 256, 0, ctx->stream>>>(ws.alpha64, (int)cols, alpha);
     SKIM_CUDA_OK(cudaGetLastError());
