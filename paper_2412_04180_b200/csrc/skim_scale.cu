@@ -44,40 +44,47 @@ struct ScaleArgs {
     int rows_per_range;
 };
 
-// Eight consecutive elements of a row starting at e0 (a multiple of 8); entries at or beyond cols come
-// back with zero importance, label 0 and alpha 1.
+// Eight consecutive elements of a row starting at e0 (a multiple of 8), as loaded; entries at or
+// beyond cols come back with zero importance, label 0 and alpha 1.
+struct Raw8 {
+    uint4 w;            // 8 binary16 weights
+    float4 ga, gb;      // 8 importances
+    uint2 l;            // 8 labels
+    double2 al[4];      // 8 alphas
+};
+
 template <bool VEC>
-__device__ __forceinline__ void load8(const ScaleArgs &a, int64_t row, int e0, float *w, float *g, int *l, double *al)
+__device__ __forceinline__ void load8(const ScaleArgs &a, int64_t row, int e0, Raw8 &r)
 {
     const uint16_t *Wr = a.W + row * a.ld;
     const float *Gr = a.G + row * a.ld;
     const uint8_t *Lr = a.labels + row * (int64_t)a.cols;
     if (VEC && e0 + 8 <= a.cols) {
-        const uint4 wv = __ldg(reinterpret_cast<const uint4 *>(Wr + e0));
-        const float4 ga = __ldg(reinterpret_cast<const float4 *>(Gr + e0)), gb = __ldg(reinterpret_cast<const float4 *>(Gr + e0 + 4));
-        const uint2 lv = __ldg(reinterpret_cast<const uint2 *>(Lr + e0));
-        const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
-        const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+        // the matrix streams through once per kernel: keep it from evicting alpha
+        r.w = __ldcs(reinterpret_cast<const uint4 *>(Wr + e0));
+        r.ga = __ldcs(reinterpret_cast<const float4 *>(Gr + e0));
+        r.gb = __ldcs(reinterpret_cast<const float4 *>(Gr + e0 + 4));
+        r.l = __ldcs(reinterpret_cast<const uint2 *>(Lr + e0));
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            w[u] = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
-            g[u] = gg[u];
-            l[u] = (int)(((u < 4 ? lv.x : lv.y) >> (8 * (u & 3))) & (KC - 1));
-        }
-#pragma unroll
-        for (int u = 0; u < 8; u += 2) {
-            const double2 av = __ldg(reinterpret_cast<const double2 *>(a.alpha + e0 + u));
-            al[u] = av.x; al[u + 1] = av.y;
-        }
+        for (int u = 0; u < 4; ++u) r.al[u] = __ldg(reinterpret_cast<const double2 *>(a.alpha + e0 + 2 * u));
     } else {
+        uint32_t ww[4] = {0u, 0u, 0u, 0u}, ll[2] = {0u, 0u};
+        float gg[8];
+        double aa[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const bool in = e0 + u < a.cols;
-            w[u] = in ? __half2float(__ushort_as_half(Wr[e0 + u])) : 0.0f;
-            g[u] = in ? Gr[e0 + u] : 0.0f;
-            l[u] = in ? (int)(Lr[e0 + u] & (KC - 1)) : 0;
-            al[u] = in ? a.alpha[e0 + u] : 1.0;
+            ww[u >> 1] |= (in ? (uint32_t)Wr[e0 + u] : 0u) << (16 * (u & 1));
+            ll[u >> 2] |= (in ? (uint32_t)(Lr[e0 + u] & (KC - 1)) : 0u) << (8 * (u & 3));
+            gg[u] = in ? Gr[e0 + u] : 0.0f;
+            aa[u] = in ? a.alpha[e0 + u] : 1.0;
         }
+        r.w = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+        r.ga = make_float4(gg[0], gg[1], gg[2], gg[3]);
+        r.gb = make_float4(gg[4], gg[5], gg[6], gg[7]);
+        r.l = make_uint2(ll[0], ll[1]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) r.al[u] = make_double2(aa[2 * u], aa[2 * u + 1]);
     }
 }
 
@@ -92,16 +99,21 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
     double *slot = slots_all + (size_t)warp * (NSUM * KC * 32) + lane;   // entry (s, k) at slot[(s * KC + k) * 32]
 #pragma unroll
     for (int q = 0; q < NSUM * KC; ++q) slot[q * 32] = 0.0;
+    // the loads of the next step are issued before the current one is worked on
+    Raw8 cur, nxt;
+    if (lane * 8 < a.cols) load8<VEC>(a, row, lane * 8, cur);
     for (int e0 = lane * 8; e0 < a.cols; e0 += 256) {
-        float w[8], g[8];
-        int l[8];
-        double al[8];
-        load8<VEC>(a, row, e0, w, g, l, al);
+        if (e0 + 256 < a.cols) load8<VEC>(a, row, e0 + 256, nxt);
+        const uint32_t ww[4] = {cur.w.x, cur.w.y, cur.w.z, cur.w.w};
+        const float g[8] = {cur.ga.x, cur.ga.y, cur.ga.z, cur.ga.w, cur.gb.x, cur.gb.y, cur.gb.z, cur.gb.w};
+        const double al[8] = {cur.al[0].x, cur.al[0].y, cur.al[1].x, cur.al[1].y, cur.al[2].x, cur.al[2].y, cur.al[3].x, cur.al[3].y};
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const double gd = (double)g[u], wd = (double)w[u];
+            const float wf = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+            const int l = (int)(((u < 4 ? cur.l.x : cur.l.y) >> (8 * (u & 3))) & (KC - 1));
+            const double gd = (double)g[u], wd = (double)wf;
             const double gw = gd * wd;
-            double *sl = slot + l[u] * 32;
+            double *sl = slot + l * 32;
             if (INIT) {
                 sl[0] += gd;
                 sl[KC * 32] += gw * wd;
@@ -111,6 +123,7 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
                 sl[2 * KC * 32] += gd * al[u] * al[u];
             }
         }
+        cur = nxt;
     }
     __syncwarp();
     // lane L adds up entry L (and L + 32) over the 32 lanes' slots, starting at its own (no bank conflicts)
@@ -148,10 +161,11 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
 template <bool VEC>
 __global__ void __launch_bounds__(GT) skim_scale_grad_kernel(ScaleArgs a)
 {
+    constexpr int RB = 8;                       // rows whose loads are in flight together
+    __shared__ double2 tq_s[RB * KC];           // their (c_k, q_k) tables
     const int j0 = (blockIdx.x * GT + threadIdx.x) * GC;
     const int64_t r0 = (int64_t)blockIdx.y * a.rows_per_range;
     const int64_t r1 = min(a.rows, r0 + a.rows_per_range);
-    if (j0 >= a.cols) return;
     double al[GC], rr[GC], acc[GC];
 #pragma unroll
     for (int u = 0; u < GC; ++u) {
@@ -161,40 +175,55 @@ __global__ void __launch_bounds__(GT) skim_scale_grad_kernel(ScaleArgs a)
         acc[u] = 0.0;
     }
     const bool full = VEC && j0 + GC <= a.cols;
-#pragma unroll 2
-    for (int64_t row = r0; row < r1; ++row) {
-        const uint16_t *Wr = a.W + row * a.ld + j0;
-        const float *Gr = a.G + row * a.ld + j0;
-        const uint8_t *Lr = a.labels + row * (int64_t)a.cols + j0;
-        float w[GC], g[GC];
-        int l[GC];
-        if (full) {
-            const uint2 wv = __ldg(reinterpret_cast<const uint2 *>(Wr));
-            const float4 gv = __ldg(reinterpret_cast<const float4 *>(Gr));
-            const uint32_t lv = __ldg(reinterpret_cast<const uint32_t *>(Lr));
-            w[0] = __half2float(__ushort_as_half((uint16_t)(wv.x & 0xffffu)));
-            w[1] = __half2float(__ushort_as_half((uint16_t)(wv.x >> 16)));
-            w[2] = __half2float(__ushort_as_half((uint16_t)(wv.y & 0xffffu)));
-            w[3] = __half2float(__ushort_as_half((uint16_t)(wv.y >> 16)));
-            g[0] = gv.x; g[1] = gv.y; g[2] = gv.z; g[3] = gv.w;
+    for (int64_t rb = r0; rb < r1; rb += RB) {
+        __syncthreads();                        // the previous batch's tables are no longer read
+        if (threadIdx.x < RB * KC && rb + threadIdx.x / KC < r1) tq_s[threadIdx.x] = a.tq[rb * KC + threadIdx.x];
+        uint2 wv[RB];
+        float4 gv[RB];
+        uint32_t lv[RB];
 #pragma unroll
-            for (int u = 0; u < GC; ++u) l[u] = (int)((lv >> (8 * u)) & (KC - 1));
-        } else {
+        for (int q = 0; q < RB; ++q) {
+            const int64_t row = rb + q;
+            wv[q] = make_uint2(0u, 0u); gv[q] = make_float4(0.f, 0.f, 0.f, 0.f); lv[q] = 0u;
+            if (row < r1 && j0 < a.cols) {
+                const uint16_t *Wr = a.W + row * a.ld + j0;
+                const float *Gr = a.G + row * a.ld + j0;
+                const uint8_t *Lr = a.labels + row * (int64_t)a.cols + j0;
+                if (full) {
+                    wv[q] = __ldcs(reinterpret_cast<const uint2 *>(Wr));
+                    gv[q] = __ldcs(reinterpret_cast<const float4 *>(Gr));
+                    lv[q] = __ldcs(reinterpret_cast<const uint32_t *>(Lr));
+                } else {
+                    uint32_t ww[2] = {0u, 0u};
+                    float gg[GC];
 #pragma unroll
-            for (int u = 0; u < GC; ++u) {
-                const bool in = j0 + u < a.cols;
-                w[u] = in ? __half2float(__ushort_as_half(Wr[u])) : 0.0f;
-                g[u] = in ? Gr[u] : 0.0f;
-                l[u] = in ? (int)(Lr[u] & (KC - 1)) : 0;
+                    for (int u = 0; u < GC; ++u) {
+                        const bool in = j0 + u < a.cols;
+                        ww[u >> 1] |= (in ? (uint32_t)Wr[u] : 0u) << (16 * (u & 1));
+                        lv[q] |= (in ? (uint32_t)(Lr[u] & (KC - 1)) : 0u) << (8 * u);
+                        gg[u] = in ? Gr[u] : 0.0f;
+                    }
+                    wv[q] = make_uint2(ww[0], ww[1]);
+                    gv[q] = make_float4(gg[0], gg[1], gg[2], gg[3]);
+                }
             }
         }
-        const double2 *tq = a.tq + row * KC;
+        __syncthreads();
 #pragma unroll
-        for (int u = 0; u < GC; ++u) {
-            const double2 cq = __ldg(tq + l[u]);
-            const double gd = (double)g[u], wd = (double)w[u];
-            const double res = wd - al[u] * cq.x;
-            acc[u] += gd * (cq.y * wd * rr[u] - 2.0 * cq.x * res);
+        for (int q = 0; q < RB; ++q) {
+            const int64_t row = rb + q;
+            if (row >= r1) break;
+            const double2 *tq = tq_s + q * KC;
+            const uint32_t ww[2] = {wv[q].x, wv[q].y};
+            const float g[GC] = {gv[q].x, gv[q].y, gv[q].z, gv[q].w};
+#pragma unroll
+            for (int u = 0; u < GC; ++u) {
+                const double2 cq = tq[(lv[q] >> (8 * u)) & (KC - 1)];
+                const double gd = (double)g[u];
+                const double wd = (double)__half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+                const double res = wd - al[u] * cq.x;
+                acc[u] += gd * (cq.y * wd * rr[u] - 2.0 * cq.x * res);
+            }
         }
     }
 #pragma unroll
