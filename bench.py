@@ -40,7 +40,7 @@ CLUSTER_BYTES_PER_ELEMENT = 6
 CLUSTER_BYTES_PER_ROW = 136
 # DRAM traffic of one launch of the dominant kernel per row, from the committed ncu capture
 # (bytes), or None when the kernel changed since the counters were taken.
-SORT_TRAFFIC_BYTES_PER_ROW = None
+SORT_TRAFFIC_BYTES_PER_ROW = 173_990   # (143.77 MB read + 212.56 MB written) / 2048 rows, profiles/skim_sort16_kernel_2048x11008.md
 DOMINANT_KERNEL = "skim_sort16_kernel"
 
 
@@ -150,6 +150,45 @@ def run_reference(args):
     }))
 
 
+def run_stage(args, ctx, stream, W, G, cent, bits, out):
+    """Times one stage outside the benchmark's step: the alpha-update (Algorithm 2, inner repeat) or the
+    consumers of the packed form, on the benchmark's matrix after one pipeline step."""
+    import torch
+    peak, peak_kind = measured_peak()
+    with torch.cuda.stream(stream):
+        if args.stage == "scale":
+            _, labels, _ = ctx.cluster_rows_at(W, G, bits, BIT_SET, ITERS, want_codes=True, centroids=cent.clone())
+            alpha = torch.ones(COLS, dtype=torch.float32, device="cuda")
+            ctx.scale_update(W, G, labels, alpha, steps=3, want_trace=False)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            trace = ctx.scale_update(W, G, labels, alpha, steps=args.steps)
+            e1.record(stream)
+            stream.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            nbytes = 2 * 7 * ROWS * COLS
+            print(json.dumps({"stage": "scale_update", "workload": WORKLOAD, "adam_steps": args.steps, "ms_per_adam_step": ms,
+                              "algorithmic_bytes_per_step": nbytes, "achieved_gbs": nbytes / (ms * 1e-3) / 1e9,
+                              "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
+                              "loss_first": float(trace[0]), "loss_last": float(trace[-1]), "kernel_launches_per_step": 3}))
+        else:
+            xq = torch.from_numpy(np.random.default_rng(1).standard_normal(COLS).astype(np.float16)).cuda()
+            wq = torch.empty((ROWS, COLS), dtype=torch.float16, device="cuda")
+            yq = torch.empty((ROWS,), dtype=torch.float32, device="cuda")
+            res = {}
+            for name, fn in (("dequantize", lambda: ctx.dequantize(out, COLS, BIT_SET, out=wq)),
+                             ("matvec", lambda: ctx.matvec(out, COLS, BIT_SET, xq, out=yq))):
+                fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(args.steps):
+                    fn()
+                e1.record(stream)
+                stream.synchronize()
+                res[name + "_ms_incl_launch_gaps"] = e0.elapsed_time(e1) / args.steps
+            print(json.dumps({"stage": "consumers", "workload": WORKLOAD, **res}))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -209,6 +248,12 @@ def run_ours(args):
     for _ in range(args.warmup):
         step()
     barrier()
+    if args.stage != "pipeline":
+        if rank == 0:
+            run_stage(args, ctx, stream, W, G, cent, bits, out)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     def busy(seconds):
         # the same steps, untimed, so that the clock samples around the timed region see this load
@@ -355,6 +400,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--rows", type=int, default=0, help="profiling only: use fewer rows of the same matrix")
+    ap.add_argument("--stage", default="pipeline", choices=["pipeline", "scale", "consumers"],
+                    help="pipeline: the benchmark proper; scale / consumers: time only the alpha-update or the "
+                         "unpacking kernels on the same matrix (their own JSON line; used for profiler captures)")
     args = ap.parse_args()
     if args.rows:
         global ROWS, WORKLOAD

@@ -256,7 +256,6 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     a.scratch = ws.cluster_scratch;
     a.rec_stride = 0;
     a.row0 = 0;
-    a.lookahead = 2 * ctx->sm_count;   // about one round of resident blocks
 
     // plan: the fp16-key sort kernel when it applies, else the generic one
     bool fast = !scaled && skim_launch_sort16(ctx, a, 0, false) == SKIM_OK;

@@ -80,15 +80,6 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
                  : "memory");
 }
 
-// Asks the L2 to fetch `bytes` (a multiple of 16, 16-byte aligned) of global memory; no data reaches the SM.
-__device__ __forceinline__ void l2_prefetch(const void *src, uint32_t bytes)
-{
-    for (uint32_t o = 0; o < bytes; o += 32768u)
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const unsigned char *>(src) + o),
-                     "r"(min(32768u, bytes - o))
-                     : "memory");
-}
-
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
@@ -162,11 +153,6 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         mbar_init(mbar, 1);
         ps.misc[0] = 0;
         ps.misc[1] = 0;
-        // the block that will run a round of blocks later finds its two rows in L2
-        if ((long long)blockIdx.x + a.lookahead < (long long)gridDim.x) {
-            l2_prefetch(Wr + (int64_t)a.lookahead * a.ld, ((uint32_t)m * 2u) & ~15u);
-            l2_prefetch(Gr + (int64_t)a.lookahead * a.ld, (uint32_t)m * 4u);
-        }
     }
     for (int d = tid; d < D0; d += THREADS) C0[d] = 0u;
     for (int d = tid; d < D1 * THREADS / 2; d += THREADS) cnt1w[d] = 0u;

@@ -81,7 +81,6 @@ struct ClusterArgs {
     unsigned char *scratch;   // row records of the current chunk (written by the sort kernel, read by the Lloyd kernel)
     long long rec_stride;     // bytes between row records
     int64_t row0;             // first row of the current chunk
-    int lookahead;            // a sort block asks the L2 for the inputs of the row this many blocks ahead
 };
 
 // Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are

@@ -179,8 +179,7 @@ int launch_unpack(skim_ctx *ctx, const UnpackArgs &a)
         attr_dev[f] = ctx->device;
         attr_smem[f] = smem;
     }
-    const int64_t want = (a.rows + UW - 1) / UW;
-    const unsigned blocks = (unsigned)(want < ctx->sm_count ? want : ctx->sm_count);   // one block per SM, rows dealt round-robin
+    const unsigned blocks = (unsigned)(a.rows < ctx->sm_count ? a.rows : ctx->sm_count);   // one block per SM, rows dealt round-robin
     skim_unpack_kernel<MATVEC><<<blocks, UT, smem, ctx->stream>>>(a);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
