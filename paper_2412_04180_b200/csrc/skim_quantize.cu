@@ -133,6 +133,13 @@ __global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
     __shared__ __half2 th_s[16];
     const int tid = threadIdx.x;
     const int64_t row = blockIdx.x;
+    const uint16_t *Wr = a.W + row * a.ld;
+    const int quad = tid >> 2, ql = tid & 3;
+    // fp16 fast path: the weights of a step are loaded one step ahead; the first load goes out
+    // before the row's parameters are read
+    const bool fast = a.vec_ok && !a.rscale;
+    uint4 ahead = make_uint4(0u, 0u, 0u, 0u);
+    if (fast && quad * 32 + ql * 8 + 8 <= a.cols) ahead = __ldg(reinterpret_cast<const uint4 *>(Wr + quad * 32 + ql * 8));
     const int pos = a.row_pos[row];
     if (pos < 0) return;
     const int b = (int)a.bits[row];
@@ -159,14 +166,14 @@ __global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
     const int64_t stride = skim_row_stride_words(a.cols, b);
     uint32_t *dst = a.packed + a.group_info[a.nb + 1 + bi] + (int64_t)(pos - a.group_info[bi]) * stride;
     const int ngroups = (int)((stride + b - 1) / b);   // a group: 32 elements -> b words
-    const uint16_t *Wr = a.W + row * a.ld;
-    const int quad = tid >> 2, ql = tid & 3;
     for (int base = 0; base < ngroups; base += PT / 4) {
         const int grp = base + quad;
         const int e0 = grp * 32 + ql * 8;
         uint32_t v = 0;
-        if (a.vec_ok && !a.rscale && e0 + 8 <= a.cols) {
-            const uint4 raw = *reinterpret_cast<const uint4 *>(Wr + e0);
+        const uint4 raw = ahead;
+        if (fast && base + PT / 4 < ngroups && e0 + (PT / 4) * 32 + 8 <= a.cols)
+            ahead = __ldg(reinterpret_cast<const uint4 *>(Wr + e0 + (PT / 4) * 32));
+        if (fast && e0 + 8 <= a.cols) {
             switch (b) {
             case 1: v = labels8_half<1>(raw, th); break;
             case 2: v = labels8_half<2>(raw, th); break;
