@@ -127,6 +127,16 @@ int skim_cluster_rows_at(skim_ctx *ctx, const uint16_t *W, const float *importan
 int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
                        double budget, uint8_t *bits, int64_t *total_bits);
 
+/*
+ * The allocation variant of the appendix on other model families (additional perplexity results):
+ * the allocation starts from the budget rounded down, floor(budget), for every row instead of from
+ * b_min, and Algorithm 1 hands out only the remaining T - rows * floor(budget) bits.  With an integer
+ * budget nothing remains: every row gets exactly that width, i.e. mixed precision is off.
+ * Arguments, tie rule, T and errors as for skim_allocate_bits.
+ */
+int skim_allocate_bits_floor(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
+                             double budget, uint8_t *bits, int64_t *total_bits);
+
 /* Packed layout (host-only helper): 32-bit words per packed row of each width,
  * ceil(cols*b/32) rounded up to a multiple of 4, and the byte size that is enough for any
  * allocation (every row at the largest width).  Outputs are host pointers; either may be NULL. */

@@ -323,6 +323,39 @@ int skim_oracle_allocate_bits(const float *err, int64_t rows, int n_bits, int b_
     return 0;
 }
 
+/*
+ * Allocation started from the floor of the budget (appendix with the results on other model
+ * families: mixed precision is switched off at integer budgets, and at non-integer ones the
+ * allocation is initialised with the budget rounded down).  Every row starts at floor(budget);
+ * Algorithm 1's loop then hands out the remaining T - rows * floor(budget) bits exactly as above.
+ */
+int skim_oracle_allocate_bits_floor(const float *err, int64_t rows, int n_bits, int b_min, double budget,
+                                    uint8_t *bits, int64_t *total)
+{
+    if (!err || !bits || rows <= 0 || n_bits <= 0 || b_min < 1) return -1;
+    int b_max = b_min + n_bits - 1;
+    if (!(budget >= (double)b_min && budget <= (double)b_max)) return -2;
+    int64_t T = (int64_t)floor((double)rows * budget + 1e-6);
+    int start = (int)floor(budget + 1e-9);
+    if (start > b_max) start = b_max;
+    int64_t K = T - rows * (int64_t)start;
+    if (K < 0 || K > rows * (int64_t)(b_max - start)) return -2;
+    for (int64_t i = 0; i < rows; ++i) bits[i] = (uint8_t)start;
+    for (int64_t step = 0; step < K; ++step) {
+        int64_t best = -1;
+        double best_gain = 0.0;
+        for (int64_t i = 0; i < rows; ++i) {
+            if (bits[i] >= b_max) continue;
+            int b = bits[i] - b_min;
+            double gain = (double)err[i * n_bits + b] - (double)err[i * n_bits + b + 1];
+            if (best < 0 || gain > best_gain) { best = i; best_gain = gain; }
+        }
+        bits[best] += 1;
+    }
+    if (total) *total = T;
+    return 0;
+}
+
 /* ------------------------------------------------------------------ emission */
 
 /* Words in one packed row of `cols` codes of `b` bits: ceil(cols*b/32), rounded up to 4 words. */

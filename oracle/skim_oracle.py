@@ -103,14 +103,15 @@ def cluster_rows(W, importance, bit_set, iters, s=None, row_bits=None, round_fp3
     return dict(centroids=centroids, codes=codes, err=err, trace=trace)
 
 
-def allocate_bits(err, b_min, budget):
-    """Greedy allocation over a float32 table [rows, n_bits]; returns (bits uint8 [rows], total)."""
+def allocate_bits(err, b_min, budget, floor_start=False):
+    """Greedy allocation over a float32 table [rows, n_bits]; returns (bits uint8 [rows], total).
+    floor_start: every row starts at floor(budget) instead of b_min."""
     err = np.ascontiguousarray(err, dtype=np.float32)
     rows, nb = err.shape
     bits = np.zeros(rows, dtype=np.uint8)
     total = C.c_int64(0)
-    rc = lib().skim_oracle_allocate_bits(_p(err), C.c_int64(rows), C.c_int(nb), C.c_int(b_min),
-                                         C.c_double(budget), _p(bits), C.byref(total))
+    fn = lib().skim_oracle_allocate_bits_floor if floor_start else lib().skim_oracle_allocate_bits
+    rc = fn(_p(err), C.c_int64(rows), C.c_int(nb), C.c_int(b_min), C.c_double(budget), _p(bits), C.byref(total))
     if rc == -2:
         raise ValueError("budget outside [b_min, b_max]")
     if rc:

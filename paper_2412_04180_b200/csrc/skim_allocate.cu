@@ -20,16 +20,16 @@ __device__ __forceinline__ unsigned long long ordered_bits(double v)
     return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// keys of one row: q[t] for t = 0 .. nb-2 (entries beyond stay 0)
-__device__ __forceinline__ void row_keys(const float *err, int64_t i, int nb, unsigned long long *q)
+// keys of one row: q[t] for t = 0 .. nb-2 (entries beyond stay 0); ld floats between rows of the table
+__device__ __forceinline__ void row_keys(const float *err, int64_t i, int ld, int nb, unsigned long long *q)
 {
     double run = 0.0;
-    float prev = __ldg(err + i * nb);
+    float prev = __ldg(err + i * ld);
 #pragma unroll
     for (int t = 0; t < SKIM_MAX_NBITS - 1; ++t) {
         q[t] = 0ull;
         if (t + 1 < nb) {
-            const float next = __ldg(err + i * nb + t + 1);
+            const float next = __ldg(err + i * ld + t + 1);
             const double gain = (double)prev - (double)next;
             run = (t == 0 || gain < run) ? gain : run;
             q[t] = ordered_bits(run);
@@ -43,7 +43,7 @@ __device__ __forceinline__ void row_keys(const float *err, int64_t i, int nb, un
 // CACHE_ROWS > 0: every thread keeps the keys of its (at most CACHE_ROWS) rows in registers for all
 // passes; CACHE_ROWS == 0: keys are recomputed from the table in every pass.
 template <int CACHE_ROWS>
-__global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restrict__ err, int64_t n, int nb,
+__global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restrict__ err, int64_t n, int ld, int nb,
                                                             int bmin, long long K, uint8_t *__restrict__ bits)
 {
     constexpr int STEPS_MAX = SKIM_MAX_NBITS - 1;
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
         for (int j = 0; j < NC; ++j) {
             const int64_t i = row_base + (int64_t)j * 32;
             unsigned long long q[SKIM_MAX_NBITS] = {0ull, 0ull, 0ull, 0ull};
-            if (j < rounds && i < n) row_keys(err, i, nb, q);
+            if (j < rounds && i < n) row_keys(err, i, ld, nb, q);
 #pragma unroll
             for (int t = 0; t < STEPS_MAX; ++t) cache[j][t] = q[t];
         }
@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
                     for (int t = 0; t < STEPS_MAX; ++t) q[t] = cache[jj][t];
                 }
         } else {
-            row_keys(err, i, nb, q);
+            row_keys(err, i, ld, nb, q);
         }
     };
 
@@ -231,13 +231,15 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
 
 }  // namespace
 
-int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int64_t K,
+int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int first_col, int64_t K,
                          uint8_t *out_bits)
 {
+    // the greedy runs on the columns first_col .. n_bits-1 of the table: every row starts at b_min + first_col
+    const int ld = bits.n_bits, nb = bits.n_bits - first_col, start = bits.b_min + first_col;
     if (rows <= 4 * AT)
-        skim_allocate_kernel<4><<<1, AT, 0, ctx->stream>>>(err, rows, bits.n_bits, bits.b_min, (long long)K, out_bits);
+        skim_allocate_kernel<4><<<1, AT, 0, ctx->stream>>>(err + first_col, rows, ld, nb, start, (long long)K, out_bits);
     else
-        skim_allocate_kernel<0><<<1, AT, 0, ctx->stream>>>(err, rows, bits.n_bits, bits.b_min, (long long)K, out_bits);
+        skim_allocate_kernel<0><<<1, AT, 0, ctx->stream>>>(err + first_col, rows, ld, nb, start, (long long)K, out_bits);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     return SKIM_OK;

@@ -201,7 +201,27 @@ int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int 
     if (total_bits) *total_bits = T;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SKIM_ERR_CUDA;
-    return skim_launch_allocate(ctx, err, rows, bits, K, bits_out);
+    return skim_launch_allocate(ctx, err, rows, bits, 0, K, bits_out);
+}
+
+int skim_allocate_bits_floor(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
+                             double budget, uint8_t *bits_out, int64_t *total_bits)
+{
+    if (!ctx || !err || !bits_out) return SKIM_ERR_NULL;
+    SkimBits bits;
+    int rc = skim_check_bits(bit_set, n_bits, &bits);
+    if (rc) return rc;
+    if (rows < 1 || rows > 0x7fffffff) return SKIM_ERR_SHAPE;
+    if (!(budget >= (double)bits.b_min && budget <= (double)bits.b_max)) return SKIM_ERR_BUDGET;
+    const int64_t T = (int64_t)floor((double)rows * budget + 1e-6);
+    int start = (int)floor(budget + 1e-9);             // every row starts at the budget rounded down
+    if (start > bits.b_max) start = bits.b_max;
+    const int64_t K = T - rows * (int64_t)start;
+    if (K < 0 || K > rows * (int64_t)(bits.b_max - start)) return SKIM_ERR_BUDGET;
+    if (total_bits) *total_bits = T;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_allocate(ctx, err, rows, bits, start - bits.b_min, K, bits_out);
 }
 
 int skim_packed_layout(int64_t rows, int64_t cols, const int *bit_set, int n_bits, int64_t *row_stride_words,

@@ -112,7 +112,7 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
                         int iters, float *centroids, uint8_t *codes, float *err);
 int skim_cluster_max_cols(int max_smem_optin, int64_t *out);
 int skim_launch_reciprocal(skim_ctx *ctx, const float *s, int64_t cols);
-int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits,
+int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int first_col,
                          int64_t K, uint8_t *out_bits);
 int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
                          const uint8_t *bits, const float *centroids, const SkimBits &bs,

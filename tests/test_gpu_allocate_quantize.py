@@ -50,6 +50,25 @@ def test_allocation_heavy_ties_and_special_tables(ctx, oracle):
             np.testing.assert_array_equal(got, want, err_msg=f"table {t} total {total}")
 
 
+@pytest.mark.parametrize("rows", [1, 33, 1000, 4096, 9000])
+def test_floor_started_allocation_matches_oracle(ctx, oracle, rows):
+    """skim_allocate_bits_floor: every row starts at floor(budget); bit-exact against the oracle's loop."""
+    err = inputs.make_error_table(rows, 4, 300 + rows, monotone=False, ties=True)
+    errd = torch.from_numpy(err).cuda()
+    for budget in (1.0, 1.25, 2.0, 2.25, 2.999, 3.0, 3.5, 4.0):
+        want, total = oracle.allocate_bits(err, 1, budget, floor_start=True)
+        got, gtotal = ctx.allocate_bits(errd, BITS, budget, floor_start=True)
+        assert gtotal == total
+        np.testing.assert_array_equal(got.cpu().numpy(), want, err_msg=f"rows={rows} budget={budget}")
+    for bit_set in ([2, 3, 4], [3, 4]):
+        sub = np.ascontiguousarray(err[:, :len(bit_set)])
+        for budget in (bit_set[0] + 0.0, bit_set[0] + 0.6, bit_set[-1] - 0.3):
+            want, total = oracle.allocate_bits(sub, bit_set[0], budget, floor_start=True)
+            got, gtotal = ctx.allocate_bits(torch.from_numpy(sub).cuda(), bit_set, budget, floor_start=True)
+            assert gtotal == total
+            np.testing.assert_array_equal(got.cpu().numpy(), want)
+
+
 @pytest.mark.parametrize("bit_set", [[2, 3], [1, 2, 3], [3, 4], [4]])
 def test_allocation_other_bit_sets(ctx, oracle, bit_set):
     err = inputs.make_error_table(777, len(bit_set), 9, monotone=False, ties=True)

@@ -76,6 +76,55 @@ def test_allocation_takes_negative_gains_when_the_budget_demands_it(oracle):
     assert list(bits) == [1, 2]
 
 
+def _brute_force_from(err, b_min, start, total):
+    """Cheapest allocation with every width >= start and the given total."""
+    rows, nb = err.shape
+    best = np.inf
+    for combo in itertools.product(range(start - b_min, nb), repeat=rows):
+        if sum(combo) + rows * b_min != total:
+            continue
+        best = min(best, sum(float(err[i, c]) for i, c in enumerate(combo)))
+    return best
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("budget", [1.0, 1.5, 2.0, 2.4, 3.0, 3.7, 4.0])
+def test_floor_started_allocation(oracle, seed, budget):
+    """Every row starts at floor(budget): an integer budget switches mixed precision off; otherwise the
+    remaining bits go greedily, which on tables with non-increasing gains is the optimum among the
+    allocations that give every row at least floor(budget) bits (brute force)."""
+    rows = 6
+    rng = np.random.default_rng(100 + seed)
+    gains = np.sort(rng.integers(1, 40, size=(rows, 3)), axis=1)[:, ::-1].astype(np.float64)
+    tail = rng.integers(1, 5, size=(rows, 1)).astype(np.float64)
+    err = np.concatenate([gains, tail], axis=1)[:, ::-1].cumsum(axis=1)[:, ::-1].astype(np.float32)
+    bits, total = oracle.allocate_bits(err, 1, budget, floor_start=True)
+    start = int(np.floor(budget + 1e-9))
+    assert total == int(np.floor(rows * budget + 1e-6)) and int(bits.sum()) == total
+    assert bits.min() >= start and bits.max() <= 4
+    if budget == start:
+        assert np.all(bits == start)
+    cost = sum(float(err[i, b - 1]) for i, b in enumerate(bits))
+    assert cost == pytest.approx(_brute_force_from(err, 1, start, total), abs=1e-9)
+    # never cheaper than the unconstrained greedy, which may leave rows below the floor
+    free, _ = oracle.allocate_bits(err, 1, budget)
+    assert cost >= sum(float(err[i, b - 1]) for i, b in enumerate(free)) - 1e-9
+
+
+def test_floor_started_allocation_hand_example(oracle):
+    # budget 7/3 = 2.33: every row starts at 2 bits, one bit is left: the gains of the third bit are
+    # 1 (row 0), 3 (row 1), 5 (row 2) -> row 2.  The plain greedy from 1 bit gives [2, 2, 3] as well here;
+    # at budget 5/3 the floor is 1 and both agree by definition.
+    err = np.array([[12, 2, 1, 0], [9, 5, 2, 0], [9, 5, 0, 0]], np.float32)
+    bits, total = oracle.allocate_bits(err, 1, 7 / 3, floor_start=True)
+    assert total == 7 and list(bits) == [2, 2, 3]
+    # a table where the floor matters: row 0 gains nothing from its second bit, the plain greedy leaves it at 1
+    err = np.array([[5, 5, 5, 5], [9, 4, 1, 0], [9, 4, 1, 0]], np.float32)
+    plain, _ = oracle.allocate_bits(err, 1, 2.0)
+    floor, _ = oracle.allocate_bits(err, 1, 2.0, floor_start=True)
+    assert list(plain) == [1, 3, 2] and list(floor) == [2, 2, 2]
+
+
 # ---------------------------------------------------------------- emission
 
 def _unpack_row(words, cols, b):
