@@ -12,6 +12,7 @@
 namespace {
 
 constexpr int AT = 1024;  // threads of the single block
+constexpr int LIST_CAP = 4096;   // live keys that fit the shared-memory list of the late passes
 
 __device__ __forceinline__ unsigned long long ordered_bits(double v)
 {
@@ -52,6 +53,11 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
     __shared__ unsigned long long s_prefix;
     __shared__ long long s_need;
     __shared__ long long wsum[AT / 32];
+    // Once few keys are still live (they share all the digits fixed so far), a pass over the table
+    // also writes them to this list, and the remaining passes look at the list only.
+    __shared__ unsigned long long list[LIST_CAP];
+    __shared__ unsigned int s_count;             // entries of the list
+    __shared__ long long s_live;                 // keys live in the coming pass
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int steps = nb - 1;
 
@@ -87,22 +93,32 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
         }
     };
 
-    if (tid == 0) { s_prefix = 0ull; s_need = K; }
+    if (tid == 0) { s_prefix = 0ull; s_need = K; s_count = 0u; s_live = (long long)n * steps; }
     for (int d = tid; d < 256; d += AT) hist[d] = 0u;
     __syncthreads();
+    bool listed = false;                         // block-uniform: the list holds every live key
 
     // radix select: after pass p the top 8(p+1) bits of the K-th largest key are known
     for (int pass = 0; pass < 8; ++pass) {
         const int shift = 56 - 8 * pass;
         const unsigned long long prefix = s_prefix;
+        if (listed) {
+            const unsigned cnt = s_count;
+            for (unsigned idx = tid; idx < cnt; idx += AT) {
+                const unsigned long long key = list[idx];
+                if ((key >> (shift + 8)) == prefix) atomicAdd(&hist[(unsigned)((key >> shift) & 0xffull)], 1u);
+            }
+        } else {
+        const bool collect = pass >= 1 && s_live <= (long long)LIST_CAP;   // block-uniform
         // Live keys share their leading bytes, so most of a warp's keys fall into one bin: the warp
         // settles on the digit of its first live key, every lane counts its keys with that digit
         // privately, and one atomic per warp adds them all; other digits are added one by one.
         bool have_digit = false;     // warp-uniform
         unsigned d0 = 0u;
         unsigned cnt0 = 0u;
-#pragma unroll 1
-        for (int j = 0; j < rounds; ++j) {
+#pragma unroll (CACHE_ROWS > 0 ? NC : 1)
+        for (int j = 0; j < (CACHE_ROWS > 0 ? NC : rounds); ++j) {
+            if (CACHE_ROWS > 0 && j >= rounds) break;
             const int64_t i = row_base + (int64_t)j * 32;
             const bool row_ok = i < n;
             unsigned long long q[SKIM_MAX_NBITS];
@@ -112,9 +128,11 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
             int first = -1;
 #pragma unroll
             for (int t = 0; t < STEPS_MAX; ++t) {
-                live[t] = row_ok && t < steps && (pass == 0 || (q[t] >> (shift + 8)) == prefix);
-                dig[t] = live[t] ? (unsigned)((q[t] >> shift) & 0xffull) : 0u;
+                const unsigned long long key = row_ok ? q[t] : 0ull;
+                live[t] = row_ok && t < steps && (pass == 0 || (key >> (shift + 8)) == prefix);
+                dig[t] = live[t] ? (unsigned)((key >> shift) & 0xffull) : 0u;
                 if (live[t] && first < 0) first = t;
+                if (collect && live[t]) list[atomicAdd(&s_count, 1u)] = key;
             }
             if (!have_digit) {
                 const unsigned any = __ballot_sync(0xffffffffu, first >= 0);
@@ -138,6 +156,8 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
         if (have_digit) {
             const unsigned total = __reduce_add_sync(0xffffffffu, cnt0);
             if (lane == 0 && total) atomicAdd(&hist[d0], total);
+        }
+        listed = collect;
         }
         __syncthreads();
         if (warp == 0) {
@@ -168,6 +188,7 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
                 }
                 s_need = need - above;
                 s_prefix = (prefix << 8) | (unsigned long long)(lane * 8 + d);
+                s_live = (long long)loc[d];
             }
         }
         __syncthreads();
@@ -177,8 +198,9 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
 
     // items equal to the threshold are taken in row-major order: count them per warp, ...
     unsigned eq_all = 0u;
-#pragma unroll 1
-    for (int j = 0; j < rounds; ++j) {
+#pragma unroll (CACHE_ROWS > 0 ? NC : 1)
+    for (int j = 0; j < (CACHE_ROWS > 0 ? NC : rounds); ++j) {
+        if (CACHE_ROWS > 0 && j >= rounds) break;
         const int64_t i = row_base + (int64_t)j * 32;
         if (i < n) {
             unsigned long long q[SKIM_MAX_NBITS];
@@ -194,8 +216,9 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
     for (int w = 0; w < warp; ++w) carry += wsum[w];
 
     // ... then rank them round by round with a warp prefix sum (rows of a round ascend with the lane)
-#pragma unroll 1
-    for (int j = 0; j < rounds; ++j) {
+#pragma unroll (CACHE_ROWS > 0 ? NC : 1)
+    for (int j = 0; j < (CACHE_ROWS > 0 ? NC : rounds); ++j) {
+        if (CACHE_ROWS > 0 && j >= rounds) break;
         const int64_t i = row_base + (int64_t)j * 32;
         const bool row_ok = i < n;
         unsigned long long q[SKIM_MAX_NBITS];
