@@ -356,6 +356,54 @@ int skim_oracle_allocate_bits_floor(const float *err, int64_t rows, int n_bits, 
     return 0;
 }
 
+/*
+ * The exact solution of the allocation problem of Section 4.2 (minimise sum_i Err(w_i, b_i) subject
+ * to the bit budget), by the dynamic programme the paper mentions and sets aside for its quadratic
+ * cost: the yardstick for Algorithm 1.  The total is fixed to the same T = floor(rows * budget + 1e-6)
+ * the greedy reaches.  With s = (bits handed out so far beyond b_min per row),
+ *   f_0(0) = 0,   f_i(s) = min_u f_{i-1}(s - u) + E[i-1][u],   u = 0 .. n_bits-1 (smallest u on ties),
+ * and the answer is f_rows(T - rows * b_min), with the widths recovered by walking the choices back.
+ *   bits out [rows];  cost out (may be NULL): the minimum, summed in row order in binary64.
+ */
+int skim_oracle_allocate_optimal(const float *err, int64_t rows, int n_bits, int b_min, double budget,
+                                 uint8_t *bits, int64_t *total, double *cost)
+{
+    if (!err || !bits || rows <= 0 || n_bits <= 0 || b_min < 1) return -1;
+    int b_max = b_min + n_bits - 1;
+    int64_t T = (int64_t)floor((double)rows * budget + 1e-6);
+    int64_t K = T - rows * (int64_t)b_min;
+    if (K < 0 || K > rows * (int64_t)(b_max - b_min)) return -2;
+    double *prev = (double *)malloc((size_t)(K + 1) * sizeof(double));
+    double *cur = (double *)malloc((size_t)(K + 1) * sizeof(double));
+    uint8_t *choice = (uint8_t *)malloc((size_t)rows * (size_t)(K + 1));
+    if (!prev || !cur || !choice) { free(prev); free(cur); free(choice); return -3; }
+    for (int64_t s = 0; s <= K; ++s) prev[s] = INFINITY;
+    prev[0] = 0.0;
+    for (int64_t i = 0; i < rows; ++i) {
+        for (int64_t s = 0; s <= K; ++s) {
+            double best = INFINITY;
+            int bu = 0;
+            for (int u = 0; u < n_bits && u <= s; ++u) {
+                double v = prev[s - u] + (double)err[i * n_bits + u];
+                if (v < best) { best = v; bu = u; }
+            }
+            cur[s] = best;
+            choice[(size_t)i * (size_t)(K + 1) + (size_t)s] = (uint8_t)bu;
+        }
+        double *t = prev; prev = cur; cur = t;
+    }
+    if (cost) *cost = prev[K];
+    int64_t s = K;
+    for (int64_t i = rows - 1; i >= 0; --i) {
+        int u = choice[(size_t)i * (size_t)(K + 1) + (size_t)s];
+        bits[i] = (uint8_t)(b_min + u);
+        s -= u;
+    }
+    free(prev); free(cur); free(choice);
+    if (total) *total = T;
+    return s == 0 ? 0 : -4;
+}
+
 /* ------------------------------------------------------------------ emission */
 
 /* Words in one packed row of `cols` codes of `b` bits: ceil(cols*b/32), rounded up to 4 words. */

@@ -119,6 +119,22 @@ def allocate_bits(err, b_min, budget, floor_start=False):
     return bits, total.value
 
 
+def allocate_optimal(err, b_min, budget):
+    """Exact minimum-error allocation with the greedy's total (dynamic programme); returns (bits, total, cost)."""
+    err = np.ascontiguousarray(err, dtype=np.float32)
+    rows, nb = err.shape
+    bits = np.zeros(rows, dtype=np.uint8)
+    total = C.c_int64(0)
+    cost = C.c_double(0.0)
+    rc = lib().skim_oracle_allocate_optimal(_p(err), C.c_int64(rows), C.c_int(nb), C.c_int(b_min), C.c_double(budget),
+                                            _p(bits), C.byref(total), C.byref(cost))
+    if rc == -2:
+        raise ValueError("budget outside [b_min, b_max]")
+    if rc:
+        raise ValueError(f"skim_oracle_allocate_optimal failed ({rc})")
+    return bits, total.value, cost.value
+
+
 def row_stride_words(cols, b):
     return int(lib().skim_oracle_row_stride_words(C.c_int64(cols), C.c_int(b)))
 

@@ -125,6 +125,35 @@ def test_floor_started_allocation_hand_example(oracle):
     assert list(plain) == [1, 3, 2] and list(floor) == [2, 2, 2]
 
 
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("budget", [1.0, 1.5, 2.2, 3.0, 3.5, 4.0])
+def test_optimal_allocation_is_the_brute_force_minimum(oracle, seed, budget):
+    """The dynamic programme against brute force over all 4^6 allocations, on tables whose gains go up and
+    down (where the greedy need not be optimal), and against the greedy itself."""
+    rows = 6
+    rng = np.random.default_rng(200 + seed)
+    err = rng.integers(0, 50, size=(rows, 4)).astype(np.float32)
+    bits, total, cost = oracle.allocate_optimal(err, 1, budget)
+    assert total == int(np.floor(rows * budget + 1e-6)) and int(bits.sum()) == total
+    assert bits.min() >= 1 and bits.max() <= 4
+    assert cost == sum(float(err[i, b - 1]) for i, b in enumerate(bits))
+    assert cost == pytest.approx(_brute_force_allocation(err, 1, total), abs=1e-9)
+    greedy, _ = oracle.allocate_bits(err, 1, budget)
+    assert cost <= sum(float(err[i, b - 1]) for i, b in enumerate(greedy)) + 1e-9
+
+
+def test_optimal_allocation_equals_greedy_cost_when_gains_do_not_increase(oracle):
+    rows = 300
+    rng = np.random.default_rng(7)
+    gains = np.sort(rng.integers(1, 1000, size=(rows, 3)), axis=1)[:, ::-1].astype(np.float64)
+    err = np.concatenate([gains, np.ones((rows, 1))], axis=1)[:, ::-1].cumsum(axis=1)[:, ::-1].astype(np.float32)
+    for budget in (1.0, 1.7, 2.5, 3.0, 3.9, 4.0):
+        bits, total, cost = oracle.allocate_optimal(err, 1, budget)
+        greedy, gtotal = oracle.allocate_bits(err, 1, budget)
+        assert total == gtotal
+        assert cost == sum(float(err[i, b - 1]) for i, b in enumerate(greedy))     # integers: exact
+
+
 # ---------------------------------------------------------------- emission
 
 def _unpack_row(words, cols, b):
