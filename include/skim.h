@@ -137,6 +137,22 @@ int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int 
 int skim_allocate_bits_floor(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
                              double budget, uint8_t *bits, int64_t *total_bits);
 
+/*
+ * The exact solution of Section 4.2's allocation problem -- minimise the summed error subject to the
+ * bit budget -- by the dynamic programme the paper names as precise but quadratic: the yardstick for
+ * Algorithm 1 (how much error the greedy leaves on the table), not a step of the quantisation path.
+ * The total is the greedy's T = floor(rows * budget + 1e-6); ties go to the smaller width.
+ * Cost: rows * (T - rows * b_min) * n_bits additions on one SM (4096 rows at 3.0 bits: a few ms).
+ *   scratch     device, 256-byte aligned, at least skim_allocate_optimal_bytes (it holds one
+ *               byte per row and state: rows * (T - rows*b_min + 1) bytes, plus two value rows)
+ *   bits        out [rows] uint8;  total_bits  host out, may be NULL
+ *   cost        device out, may be NULL: the minimum, one binary64 (the errors added in row order)
+ */
+int skim_allocate_optimal_bytes(int64_t rows, const int *bit_set, int n_bits, double budget, size_t *out);
+int skim_allocate_optimal(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
+                          double budget, void *scratch, size_t scratch_bytes, uint8_t *bits,
+                          int64_t *total_bits, double *cost);
+
 /* Packed layout (host-only helper): 32-bit words per packed row of each width,
  * ceil(cols*b/32) rounded up to a multiple of 4, and the byte size that is enough for any
  * allocation (every row at the largest width).  Outputs are host pointers; either may be NULL. */

@@ -252,7 +252,73 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
     }
 }
 
+// Exact allocation (the dynamic programme Section 4.2 mentions as the precise but quadratic solution):
+// f_i(s) = min_u f_{i-1}(s - u) + E[i-1][u] over s = bits handed out beyond b_min, smallest u on ties; one
+// block walks the rows, its threads share the states; the choices are kept to walk back from s = K.
+__global__ void __launch_bounds__(AT) skim_allocate_optimal_kernel(const float *__restrict__ err, int64_t n, int nb,
+                                                                    int bmin, long long K, double *fa, double *fb,
+                                                                    uint8_t *choice, uint8_t *__restrict__ bits,
+                                                                    double *cost)
+{
+    const int tid = threadIdx.x;
+    const double INF = __longlong_as_double(0x7ff0000000000000ll);
+    for (long long s = tid; s <= K; s += AT) { fa[s] = INF; fb[s] = INF; }
+    __syncthreads();
+    if (tid == 0) fa[0] = 0.0;
+    __syncthreads();
+    double *prev = fa, *cur = fb;
+    for (int64_t i = 0; i < n; ++i) {
+        double e[SKIM_MAX_NBITS];
+#pragma unroll
+        for (int u = 0; u < SKIM_MAX_NBITS; ++u) e[u] = u < nb ? (double)__ldg(err + i * nb + u) : 0.0;
+        const long long top = min(K, (long long)(i + 1) * (nb - 1));     // states beyond are unreachable (and stay infinite)
+        uint8_t *ch = choice + (size_t)i * (size_t)(K + 1);
+        for (long long s = tid; s <= top; s += AT) {
+            double best = INF;
+            int bu = 0;
+#pragma unroll
+            for (int u = 0; u < SKIM_MAX_NBITS; ++u) {
+                if (u < nb && u <= s) {
+                    const double v = prev[s - u] + e[u];
+                    if (v < best) { best = v; bu = u; }
+                }
+            }
+            cur[s] = best;
+            ch[s] = (uint8_t)bu;
+        }
+        __syncthreads();
+        double *t = prev; prev = cur; cur = t;
+    }
+    if (tid == 0) {
+        if (cost) *cost = prev[K];
+        long long s = K;
+        for (int64_t i = n - 1; i >= 0; --i) {
+            const int u = choice[(size_t)i * (size_t)(K + 1) + (size_t)s];
+            bits[i] = (uint8_t)(bmin + u);
+            s -= u;
+        }
+    }
+}
+
 }  // namespace
+
+size_t skim_allocate_optimal_scratch(int64_t rows, int64_t K)
+{
+    const size_t f = skim_align256((size_t)(K + 1) * sizeof(double));
+    return 2 * f + skim_align256((size_t)rows * (size_t)(K + 1));
+}
+
+int skim_launch_allocate_optimal(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int64_t K,
+                                 void *scratch, uint8_t *out_bits, double *cost)
+{
+    const size_t f = skim_align256((size_t)(K + 1) * sizeof(double));
+    unsigned char *p = (unsigned char *)scratch;
+    skim_allocate_optimal_kernel<<<1, AT, 0, ctx->stream>>>(err, rows, bits.n_bits, bits.b_min, (long long)K, (double *)p,
+                                                           (double *)(p + f), p + 2 * f, out_bits, cost);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    return SKIM_OK;
+}
 
 int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int first_col, int64_t K,
                          uint8_t *out_bits)

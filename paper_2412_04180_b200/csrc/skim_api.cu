@@ -224,6 +224,47 @@ int skim_allocate_bits_floor(skim_ctx *ctx, const float *err, int64_t rows, cons
     return skim_launch_allocate(ctx, err, rows, bits, start - bits.b_min, K, bits_out);
 }
 
+namespace {
+int optimal_plan(int64_t rows, const int *bit_set, int n_bits, double budget, SkimBits *bits, int64_t *T, int64_t *K)
+{
+    int rc = skim_check_bits(bit_set, n_bits, bits);
+    if (rc) return rc;
+    if (rows < 1 || rows > 0x7fffffff) return SKIM_ERR_SHAPE;
+    if (!(budget >= (double)bits->b_min && budget <= (double)bits->b_max)) return SKIM_ERR_BUDGET;
+    *T = (int64_t)floor((double)rows * budget + 1e-6);
+    *K = *T - rows * (int64_t)bits->b_min;
+    if (*K < 0 || *K > rows * (int64_t)(bits->b_max - bits->b_min)) return SKIM_ERR_BUDGET;
+    return SKIM_OK;
+}
+}  // namespace
+
+int skim_allocate_optimal_bytes(int64_t rows, const int *bit_set, int n_bits, double budget, size_t *out)
+{
+    if (!out) return SKIM_ERR_NULL;
+    SkimBits bits;
+    int64_t T, K;
+    int rc = optimal_plan(rows, bit_set, n_bits, budget, &bits, &T, &K);
+    if (rc) return rc;
+    *out = skim_allocate_optimal_scratch(rows, K);
+    return SKIM_OK;
+}
+
+int skim_allocate_optimal(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits, double budget,
+                          void *scratch, size_t scratch_bytes, uint8_t *bits_out, int64_t *total_bits, double *cost)
+{
+    if (!ctx || !err || !bits_out || !scratch) return SKIM_ERR_NULL;
+    SkimBits bits;
+    int64_t T, K;
+    int rc = optimal_plan(rows, bit_set, n_bits, budget, &bits, &T, &K);
+    if (rc) return rc;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0 || scratch_bytes < skim_allocate_optimal_scratch(rows, K))
+        return SKIM_ERR_WORKSPACE;
+    if (total_bits) *total_bits = T;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_allocate_optimal(ctx, err, rows, bits, K, scratch, bits_out, cost);
+}
+
 int skim_packed_layout(int64_t rows, int64_t cols, const int *bit_set, int n_bits, int64_t *row_stride_words,
                        size_t *max_packed_bytes)
 {

@@ -114,6 +114,9 @@ int skim_cluster_max_cols(int max_smem_optin, int64_t *out);
 int skim_launch_reciprocal(skim_ctx *ctx, const float *s, int64_t cols);
 int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int first_col,
                          int64_t K, uint8_t *out_bits);
+size_t skim_allocate_optimal_scratch(int64_t rows, int64_t K);
+int skim_launch_allocate_optimal(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int64_t K,
+                                 void *scratch, uint8_t *out_bits, double *cost);
 int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld,
                          const uint8_t *bits, const float *centroids, const SkimBits &bs,
                          uint32_t *packed, int32_t *row_order, int64_t *group_info, uint16_t *lut);

@@ -20,7 +20,7 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
              -7: "SKIM_ERR_BAD_DATA", -8: "SKIM_ERR_SCALE", -9: "SKIM_ERR_ALIGN", -10: "SKIM_ERR_STATIC_LIMIT"}
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
-           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor",
+           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
            "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
            "skim_kernel_times", "skim_strerror"]
@@ -180,6 +180,23 @@ class Skim:
         _chk(fn(self._h, _ptr(err), C.c_int64(rows), arr, C.c_int(nb), C.c_double(budget), _ptr(bits), C.byref(total)),
              "skim_allocate_bits_floor" if floor_start else "skim_allocate_bits")
         return bits, total.value
+
+    def allocate_optimal(self, err, bit_set, budget):
+        """Exact minimum-error allocation (dynamic programme); returns (bits uint8 [rows], total_bits, cost)."""
+        _dev(err, torch.float32, "err")
+        rows = err.shape[0]
+        arr, nb, _ = _bits(bit_set)
+        need = C.c_size_t()
+        _chk(lib().skim_allocate_optimal_bytes(C.c_int64(rows), arr, C.c_int(nb), C.c_double(budget), C.byref(need)),
+             "skim_allocate_optimal_bytes")
+        scratch = torch.empty(need.value, dtype=torch.uint8, device=err.device)
+        bits = torch.empty((rows,), dtype=torch.uint8, device=err.device)
+        cost = torch.zeros((1,), dtype=torch.float64, device=err.device)
+        total = C.c_int64()
+        _chk(lib().skim_allocate_optimal(self._h, _ptr(err), C.c_int64(rows), arr, C.c_int(nb), C.c_double(budget),
+                                         _ptr(scratch), C.c_size_t(need.value), _ptr(bits), C.byref(total), _ptr(cost)),
+             "skim_allocate_optimal")
+        return bits, total.value, float(cost.item())
 
     @staticmethod
     def packed_layout(rows, cols, bit_set):

@@ -69,6 +69,27 @@ def test_floor_started_allocation_matches_oracle(ctx, oracle, rows):
             np.testing.assert_array_equal(got.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("rows", [1, 7, 300, 2000])
+def test_optimal_allocation_matches_oracle(ctx, oracle, rows):
+    """skim_allocate_optimal: same recurrence, same order of additions, same tie rule as the oracle's dynamic
+    programme, so widths and cost are bit-identical; the greedy never beats it."""
+    err = inputs.make_error_table(rows, 4, 500 + rows, monotone=False, ties=True)
+    errd = torch.from_numpy(err).cuda()
+    for budget in (1.0, 1.4, 2.25, 3.0, 3.6, 4.0):
+        want, total, cost = oracle.allocate_optimal(err, 1, budget)
+        got, gtotal, gcost = ctx.allocate_optimal(errd, BITS, budget)
+        assert gtotal == total and gcost == cost
+        np.testing.assert_array_equal(got.cpu().numpy(), want, err_msg=f"rows={rows} budget={budget}")
+        greedy, _ = ctx.allocate_bits(errd, BITS, budget)
+        gsum = float(err[np.arange(rows), greedy.cpu().numpy().astype(np.int64) - 1].astype(np.float64).sum())
+        assert gcost <= gsum * (1 + 1e-12) + 1e-300
+    sub = np.ascontiguousarray(err[:, :2])
+    want, total, cost = oracle.allocate_optimal(sub, 3, 3.5)
+    got, gtotal, gcost = ctx.allocate_optimal(torch.from_numpy(sub).cuda(), [3, 4], 3.5)
+    assert gtotal == total and gcost == cost
+    np.testing.assert_array_equal(got.cpu().numpy(), want)
+
+
 @pytest.mark.parametrize("bit_set", [[2, 3], [1, 2, 3], [3, 4], [4]])
 def test_allocation_other_bit_sets(ctx, oracle, bit_set):
     err = inputs.make_error_table(777, len(bit_set), 9, monotone=False, ties=True)
