@@ -45,7 +45,7 @@ struct SkimWorkspace {
     double *alpha64;             // [cols]     scale-update master copy of alpha
     double *adam_m;              // [cols]
     double *adam_v;              // [cols]
-    double *ralpha;              // [cols]     (unused)
+    double *ralpha;              // [cols]     (reserved)
     double *loss_part;           // [rows]     scale update: loss of every row
     double *grad_part;           // [SKIM_SCALE_MAX_CTAS][cols]  partial gradients of the row ranges
     double *scale_const;         // [rows][16][2]  scale update: per-cluster constants (sum g, sum g w^2)
