@@ -88,19 +88,19 @@ struct ClusterArgs {
 //   hdr     int nd (number of distinct values) at byte 0; float dvals[16] at byte 64
 //   seg     one 32-byte entry per segment of 64 groups (512 elements): the binary64 sums of g,
 //           g*x and g*x^2 over all earlier segments; entry nseg holds the row totals
-//   groups  one 80-byte record per group of 8 sorted elements: 8 values, 8 importances, and the
-//           binary64 sums of g and g*x from the start of the group's segment to the group's first
-//           element: with the segment entry, everything a boundary needs in one Lloyd iteration.
-//           The last group is padded with the largest finite value and zero importance.
+//   groups  one 96-byte record per group of 8 sorted elements, three whole 32-byte sectors: the 8
+//           values | the 8 importances | the binary64 sums of g, g*x and g*x^2 from the start of
+//           the group's segment to the group's first element (and 8 bytes of padding).  With the
+//           segment entry that is everything a boundary needs in one Lloyd iteration.  The last
+//           group is padded with the largest finite value and zero importance.  Every sector is
+//           written by one 32-byte store and never touched again.
 //   gi      group index: first value of every group, sk_entries(m) floats (padded likewise)
-//   p2      binary64 sums of g*x^2 from the segment start to every group start (ngrp entries),
-//           read once, for the error
 struct RowRecord {
-    size_t seg, groups, gi, p2, total;
-    size_t gi_bytes, p2_bytes;
+    size_t seg, groups, gi, total;
+    size_t gi_bytes;
     int ngrp, nseg;
 };
-constexpr int SKIM_GROUP_BYTES = 80;
+constexpr int SKIM_GROUP_BYTES = 96;                // three 32-byte sectors
 constexpr int SKIM_SEG_SHIFT = 6;                   // a segment is 64 groups (512 elements)
 constexpr float SKIM_PAD_VALUE = 3.402823466e38f;   // largest finite binary32: 0 * padding stays 0
 
@@ -112,12 +112,10 @@ __host__ __device__ inline RowRecord row_record(int m)
     R.ngrp = (m + 7) >> 3;
     R.nseg = (R.ngrp + (1 << SKIM_SEG_SHIFT) - 1) >> SKIM_SEG_SHIFT;
     R.gi_bytes = (size_t)sk_entries(m) * 4;
-    R.p2_bytes = ((size_t)R.ngrp * 8 + 15) & ~(size_t)15;
     size_t off = 128;
     R.seg = off; off += (size_t)(R.nseg + 1) * 32;
     R.groups = off; off += (size_t)R.ngrp * SKIM_GROUP_BYTES;
     R.gi = off; off += R.gi_bytes;
-    R.p2 = off; off += R.p2_bytes;
     R.total = (off + 127) & ~(size_t)127;
     return R;
 }
@@ -129,6 +127,18 @@ __device__ __forceinline__ void copy16(void *dst, const void *src, size_t bytes)
     uint4 *d = reinterpret_cast<uint4 *>(dst);
     const uint4 *s = reinterpret_cast<const uint4 *>(src);
     for (size_t i = threadIdx.x; i < bytes / 16; i += THREADS) d[i] = s[i];
+}
+
+// One 32-byte store to a 32-byte aligned global address (a whole sector in one instruction).
+__device__ __forceinline__ void st_sector(void *p, const float *v)
+{
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+                 "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                 : "memory");
+}
+__device__ __forceinline__ void st_sector(void *p, double a, double b, double c)
+{
+    asm volatile("st.global.v4.f64 [%0], {%1, %2, %3, %4};" ::"l"(p), "d"(a), "d"(b), "d"(c), "d"(0.0) : "memory");
 }
 
 // The sorted row as the record pass sees it.  A source gives the keys and importances of one group
@@ -196,7 +206,6 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
     const int m = a.m;
     const RowRecord R = row_record(m);
     unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
-    double *p2 = reinterpret_cast<double *>(rec + R.p2);
     float *gi = reinterpret_cast<float *>(rec + R.gi);
     int distinct = 0;
     unsigned bad = 0u;
@@ -223,11 +232,9 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
                         prev = ks[u];
                     }
                 }
-                float4 *d = reinterpret_cast<float4 *>(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES);
-                d[0] = make_float4(x[0], x[1], x[2], x[3]);
-                d[1] = make_float4(x[4], x[5], x[6], x[7]);
-                d[2] = make_float4(gs[0], gs[1], gs[2], gs[3]);
-                d[3] = make_float4(gs[4], gs[5], gs[6], gs[7]);
+                unsigned char *gr = rec + R.groups + (size_t)q * SKIM_GROUP_BYTES;
+                st_sector(gr, x);
+                st_sector(gr + 32, gs);
                 first[h] = x[0];
                 double t0[8], t1[8], t2[8];
 #pragma unroll
@@ -264,8 +271,7 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
         for (int h = 0; h < 2; ++h) {
             const int q = q0 + h;
             if (q < R.ngrp) {
-                *reinterpret_cast<double2 *>(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES + 64) = make_double2(e0, e1);
-                p2[q] = e2;
+                st_sector(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES + 64, e0, e1, e2);
                 gi[q] = first[h];
             }
             e0 += a0; e1 += a1; e2 += a2;

@@ -57,12 +57,12 @@ struct SkimWorkspace {
 #define SKIM_SCALE_MAX_CTAS 296
 #define SKIM_CLUSTER_CHUNK_ROWS 8192   // rows clustered per sort-kernel / Lloyd-kernel pair
 
-// Upper bound of one row record of the clustering (4-byte keys): 128-byte header, 80 bytes per
-// group of 8 elements, group index 0.5 B and one prefix sum 1 B per element, plus rounding.
+// Upper bound of one row record of the clustering: 128-byte header, 96 bytes per group of 8
+// elements, group index 0.5 B per element, segment table, plus rounding.
 __host__ __device__ static inline size_t skim_cluster_record_bytes(int64_t cols)
 {
     const size_t m8 = ((size_t)cols + 7) & ~(size_t)7;
-    return (12 * m8 + 1024 + 127) & ~(size_t)127;
+    return (13 * m8 + 1024 + 127) & ~(size_t)127;
 }
 
 static inline size_t skim_align256(size_t v) { return (v + 255) & ~(size_t)255; }

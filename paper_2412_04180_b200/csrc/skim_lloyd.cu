@@ -32,7 +32,7 @@ struct Group {
     {
         const float4 *q = reinterpret_cast<const float4 *>(gr);
         xa = __ldg(q); xb = __ldg(q + 1); ga = __ldg(q + 2); gb = __ldg(q + 3);
-        p = __ldg(reinterpret_cast<const double2 *>(gr + 64));
+        p = __ldg(reinterpret_cast<const double2 *>(gr + 64));   // the g*x^2 sum at +80 is read once, for the error
     }
     // number of values <= t (values ascend; the padding is the largest finite value)
     __device__ __forceinline__ int count_le(float t) const
@@ -121,7 +121,6 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
     const int m = a.m;
     const RowRecord R = row_record(m);
     const unsigned char *groups = rec + R.groups;
-    const double *P2 = reinterpret_cast<const double *>(rec + R.p2);
     const double4 *seg = reinterpret_cast<const double4 *>(rec + R.seg);   // 32-byte entries; a few hot lines, served by L1
     const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
     const float INF = __int_as_float(0x7f800000);
@@ -190,7 +189,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 P0 = sb.x + grp.p.x;
                 P1 = sb.y + grp.p.y;
                 if (final) {
-                    Pc = __ldg(&seg[grp_i >> SKIM_SEG_SHIFT].z) + __ldg(P2 + grp_i);
+                    Pc = __ldg(&seg[grp_i >> SKIM_SEG_SHIFT].z) + __ldg(reinterpret_cast<const double *>(groups + (size_t)grp_i * SKIM_GROUP_BYTES + 80));
                     add_group<true>(grp, cntk, P0, P1, Pc);
                 } else {
                     add_group<false>(grp, cntk, P0, P1, Pc);
