@@ -272,10 +272,12 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
             const int q = q0 + h;
             if (q < R.ngrp) {
                 st_sector(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES + 64, e0, e1, e2);
-                gi[q] = first[h];
             }
             e0 += a0; e1 += a1; e2 += a2;
         }
+        // the two groups' entries of the group index, as one store (q0 is even)
+        if (q0 + 1 < R.ngrp) *reinterpret_cast<float2 *>(gi + q0) = make_float2(first[0], first[1]);
+        else if (q0 < R.ngrp) gi[q0] = first[0];
     }
     if (bad) atomicOr(a.status, (unsigned long long)bad);
     for (int q = R.ngrp + threadIdx.x; q < sk_entries(m); q += THREADS) gi[q] = SKIM_PAD_VALUE;

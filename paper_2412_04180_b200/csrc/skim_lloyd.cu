@@ -24,14 +24,23 @@ struct LloydSmem {
     float dvals[16];
 };
 
+// One 32-byte read-only load from a 32-byte aligned global address.
+__device__ __forceinline__ void ld_sector(const unsigned char *p, float4 &a, float4 &b)
+{
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w)
+                 : "l"(p));
+}
+
 // One group record in registers.
 struct Group {
     float4 xa, xb, ga, gb;
     double2 p;   // prefix sums of g and g*x at the group's first element
     __device__ __forceinline__ void load(const unsigned char *gr)
     {
-        const float4 *q = reinterpret_cast<const float4 *>(gr);
-        xa = __ldg(q); xb = __ldg(q + 1); ga = __ldg(q + 2); gb = __ldg(q + 3);
+        // the record is three 32-byte sectors: values, importances, sums; one read-only load each
+        ld_sector(gr, xa, xb);
+        ld_sector(gr + 32, ga, gb);
         p = __ldg(reinterpret_cast<const double2 *>(gr + 64));   // the g*x^2 sum at +80 is read once, for the error
     }
     // number of values <= t (values ascend; the padding is the largest finite value)
