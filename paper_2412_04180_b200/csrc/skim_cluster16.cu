@@ -5,7 +5,8 @@
 // and the sort moves one 32-bit word per element: (key << 16) | column.
 //
 //   load    128-bit loads of the fp16 row straight into keys.
-//   pass 0  low 12 key bits, 4096 block-wide counters, slots claimed with shared-memory atomics.
+//   pass 0  low 12 key bits, 4096 block-wide counters; the counting atomic already hands every item
+//           its slot inside its bin.
 //           The first pass of an LSD sort need not be stable, so no ranking is needed.  The
 //           scatter also counts, per owner thread of pass 1 and high digit, how many items land
 //           in that thread's stretch of positions.
@@ -184,8 +185,9 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
             if (real && (h & 0x7c00u) == 0x7c00u) bad |= 1u;
             if (h == 0x8000u) h = 0;                      // -0 and +0 are one value
             const uint32_t key = (uint32_t)K::from_half_bits(h);
-            item[j * 8 + u] = real ? ((key << 16) | (uint32_t)(e0 + u)) : NO_ITEM;
-            if (real) atomicAdd(&C0[key & (D0 - 1)], 1u);
+            // the count's old value is the item's slot inside its bin; it rides in the low half until the
+            // scatter puts the column there (the column follows from the item's place in the thread)
+            item[j * 8 + u] = real ? ((key << 16) | atomicAdd(&C0[key & (D0 - 1)], 1u)) : NO_ITEM;
         }
     }
     if (bad) atomicOr(a.status, (unsigned long long)bad);
@@ -217,8 +219,9 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     for (int i = 0; i < ITEMS; ++i) {
         if (item[i] != NO_ITEM) {
             const uint32_t key = item[i] >> 16;
-            const uint32_t pos = atomicAdd(&C0[key & (D0 - 1)], 1u);
-            buf[pos] = item[i];
+            const uint32_t pos = C0[key & (D0 - 1)] + (item[i] & 0xffffu);      // bin base + slot
+            const uint32_t col = (uint32_t)(((i >> 3) * THREADS + tid) * 8 + (i & 7));
+            buf[pos] = (key << 16) | col;
             // one more item of digit key >> 12 in the stretch of pass-1 owner pos / ITEMS
             const uint32_t owner = pos / ITEMS;
             atomicAdd(&cnt1w[((key >> D0_BITS) * THREADS + owner) >> 1], (owner & 1u) ? 0x10000u : 1u);
