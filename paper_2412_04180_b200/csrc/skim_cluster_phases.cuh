@@ -86,7 +86,7 @@ struct ClusterArgs {
 // Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are
 // multiples of 16 bytes; values are binary32 whatever key type sorted the row.
 //   hdr     int nd (number of distinct values) at byte 0; float dvals[16] at byte 64
-//   seg     one 32-byte entry per segment of 64 groups (512 elements): the binary64 sums of g,
+//   seg     one 32-byte entry per segment of 32 groups (256 elements): the binary64 sums of g,
 //           g*x and g*x^2 over all earlier segments; entry nseg holds the row totals
 //   groups  one 96-byte record per group of 8 sorted elements, three whole 32-byte sectors: the 8
 //           values | the 8 importances | the binary64 sums of g, g*x and g*x^2 from the start of
@@ -101,7 +101,7 @@ struct RowRecord {
     int ngrp, nseg;
 };
 constexpr int SKIM_GROUP_BYTES = 96;                // three 32-byte sectors
-constexpr int SKIM_SEG_SHIFT = 6;                   // a segment is 64 groups (512 elements)
+constexpr int SKIM_SEG_SHIFT = 5;                   // a segment is 32 groups (256 elements): one group per lane of a warp
 constexpr float SKIM_PAD_VALUE = 3.402823466e38f;   // largest finite binary32: 0 * padding stays 0
 
 __host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
@@ -161,7 +161,7 @@ template <typename KeyT> struct SortedArrays {
 
 // Small per-block scratch of the phases below.
 struct PhaseSmem {
-    double segtot[64][3];   // sums of every segment of 64 groups (rows of up to 24 576 elements have 48)
+    double segtot[96][3];   // sums of every segment (rows of up to 24 576 elements have 96 segments of 32 groups)
     float tfs[32];     // scratch of collect_distinct
     float dvals[32];   // the row's distinct values when there are at most 16
     int misc[4];       // [0] distinct count, [1] slot counter
@@ -190,7 +190,7 @@ __device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, 
 }
 
 // Writes the row record from the sorted row (a source, see above; padded to whole groups: largest
-// key / zero importance).  One pass: a lane takes two adjacent groups of 8 elements, decodes them,
+// key / zero importance).  One pass: a lane takes 2^(SKIM_SEG_SHIFT - 5) adjacent groups of 8 elements (one, as measured best), decodes them,
 // stores their values and importances, sums g, g*x, g*x^2 in binary64 (pairwise); one warp scan over
 // the lanes' totals turns the 64 group sums of a segment into prefix sums, which complete the
 // group records in global memory.  Segments are independent, so no warp waits for another.
@@ -210,12 +210,13 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
     int distinct = 0;
     unsigned bad = 0u;
     for (int sgm = warp; sgm < R.nseg; sgm += NW) {
-        const int q0 = (sgm << SKIM_SEG_SHIFT) + 2 * lane;
+        constexpr int GPL = 1 << (SKIM_SEG_SHIFT - 5);        // groups per lane
+        const int q0 = (sgm << SKIM_SEG_SHIFT) + GPL * lane;
         double a0 = 0.0, a1 = 0.0, a2 = 0.0;       // sums of the lane's first group
         double w0 = 0.0, w1 = 0.0, w2 = 0.0;       // sums of both
         float first[2] = {0.0f, 0.0f};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < GPL; ++h) {
             const int q = q0 + h;
             if (q < R.ngrp) {
                 const int e = q << 3;
@@ -268,7 +269,7 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
         if (lane == 31) { ps.segtot[sgm][0] = i0; ps.segtot[sgm][1] = i1; ps.segtot[sgm][2] = i2; }
         double e0 = i0 - w0, e1 = i1 - w1, e2 = i2 - w2;     // sums from the segment start to the lane's first group
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < GPL; ++h) {
             const int q = q0 + h;
             if (q < R.ngrp) {
                 st_sector(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES + 64, e0, e1, e2);
@@ -276,7 +277,7 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
             e0 += a0; e1 += a1; e2 += a2;
         }
         // the two groups' entries of the group index, as one store (q0 is even)
-        if (q0 + 1 < R.ngrp) *reinterpret_cast<float2 *>(gi + q0) = make_float2(first[0], first[1]);
+        if (GPL == 2 && q0 + 1 < R.ngrp) *reinterpret_cast<float2 *>(gi + q0) = make_float2(first[0], first[1]);
         else if (q0 < R.ngrp) gi[q0] = first[0];
     }
     if (bad) atomicOr(a.status, (unsigned long long)bad);
