@@ -192,7 +192,7 @@ __device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, 
 // Writes the row record from the sorted row (a source, see above; padded to whole groups: largest
 // key / zero importance).  One pass: a lane takes 2^(SKIM_SEG_SHIFT - 5) adjacent groups of 8 elements (one, as measured best), decodes them,
 // stores their values and importances, sums g, g*x, g*x^2 in binary64 (pairwise); one warp scan over
-// the lanes' totals turns the 64 group sums of a segment into prefix sums, which complete the
+// the lanes' totals turns the group sums of a segment into prefix sums, which complete the
 // group records in global memory.  Segments are independent, so no warp waits for another.
 // Afterwards one warp turns the segment sums into the segment table.  Call with all threads.
 // COUNT: the pass also counts the row's distinct values (ps.misc[0..1] zeroed before, and synced)
