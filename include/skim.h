@@ -84,7 +84,7 @@ int skim_max_cols(const skim_ctx *ctx, int64_t *out);
 /* Bytes of device scratch needed for matrices of up to rows x cols; `out` is a host pointer.
  * The workspace must be 256-byte aligned and stays owned by the caller.  It also stores the
  * installed scale vector, so it must outlive every call that follows skim_apply_scale.  Most of
- * it is the clustering's scratch: about 12 bytes per element for min(rows, 8192) rows (the sorted
+ * it is the clustering's scratch: about 13 bytes per element for min(rows, 8192) rows (the sorted
  * rows with their prefix sums, which the sort kernel hands to the Lloyd kernel); the scale update
  * adds 8 bytes x 296 x cols of partial gradients and 520 bytes per row. */
 int skim_workspace_bytes(int64_t rows, int64_t cols, size_t *out);
