@@ -7,7 +7,7 @@
 // single row cannot go fast; the kernel gets its throughput from the number of rows in flight: up to 32
 // warps per SM, each on its own row.  A warp first copies its row's group index (4 bytes per 8
 // elements) into shared memory, so that the boundary search never waits on global memory; per
-// iteration a lane then reads one 80-byte group record through the read-only path, the one global
+// iteration a lane then reads one 96-byte group record through the read-only path, the one global
 // round trip of the iteration.
 #include "skim_cluster_phases.cuh"
 
@@ -155,6 +155,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
     float tf = INF;                                   // no boundary above the last centroid
     double err_j = 0.0;
     int gprev = -1;                                   // group of the previous boundary position
+    int gstep = 0;                                    // its last move: boundaries keep drifting the same way
     for (int it = 0;; ++it) {
         const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
         int B = m, grp_i = 0, cntk = 0;
@@ -169,7 +170,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
             int nle = -1;                              // group-index entries <= tf
             if (gprev >= 0) {
                 Window win;
-                win.load(gi, ngi, gprev + 1);
+                win.load(gi, ngi, gprev + 1 + gstep);     // centred where the boundary is heading
                 const int cnt = win.count_le(tf);
                 if ((cnt > 0 || win.ws == 0) && cnt < WIN) nle = win.ws + cnt;
             }
@@ -182,6 +183,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 nle = lo;
             }
             grp_i = max(nle - 1, 0);
+            gstep = gprev >= 0 ? grp_i - gprev : 0;
             gprev = grp_i;
             const unsigned char *gr = groups + (size_t)grp_i * SKIM_GROUP_BYTES;
             grp.load(gr);
