@@ -45,7 +45,6 @@ struct SkimWorkspace {
     double *alpha64;             // [cols]     scale-update master copy of alpha
     double *adam_m;              // [cols]
     double *adam_v;              // [cols]
-    double *ralpha;              // [cols]     (reserved)
     double *loss_part;           // [rows]     scale update: loss of every row
     double *grad_part;           // [SKIM_SCALE_MAX_CTAS][cols]  partial gradients of the row ranges
     double *scale_const;         // [rows][16][2]  scale update: per-cluster constants (sum g, sum g w^2)
@@ -79,7 +78,6 @@ static inline SkimWorkspace skim_carve(void *base, int64_t rows, int64_t cols)
     w.alpha64 = (double *)take((size_t)cols * 8);
     w.adam_m = (double *)take((size_t)cols * 8);
     w.adam_v = (double *)take((size_t)cols * 8);
-    w.ralpha = (double *)take((size_t)cols * 8);
     w.loss_part = (double *)take((size_t)(rows > SKIM_SCALE_MAX_CTAS ? rows : SKIM_SCALE_MAX_CTAS) * 8);
     w.grad_part = (double *)take((size_t)SKIM_SCALE_MAX_CTAS * (size_t)cols * 8);
     w.scale_const = (double *)take((size_t)rows * 16 * 2 * 8);
