@@ -131,6 +131,15 @@ int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int 
                        double budget, uint8_t *bits, int64_t *total_bits);
 
 /*
+ * Algorithm 1 with its stopping rule as printed: bits are handed out until the total reaches
+ * rows * budget, so a non-integer product is rounded UP, T = ceil(rows * budget - 1e-6), and the
+ * average may exceed the budget by less than 1/rows of a bit.  Otherwise as skim_allocate_bits, which
+ * rounds down to keep Section 4.2's constraint (average <= budget).
+ */
+int skim_allocate_bits_until(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
+                             double budget, uint8_t *bits, int64_t *total_bits);
+
+/*
  * The allocation variant of the appendix on other model families (additional perplexity results):
  * the allocation starts from the budget rounded down, floor(budget), for every row instead of from
  * b_min, and Algorithm 1 hands out only the remaining T - rows * floor(budget) bits.  With an integer

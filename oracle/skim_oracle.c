@@ -324,6 +324,37 @@ int skim_oracle_allocate_bits(const float *err, int64_t rows, int n_bits, int b_
 }
 
 /*
+ * Algorithm 1 with its stopping rule taken literally: bits are handed out "until sum_i b_i >= n * bit",
+ * so a non-integer n * bit is rounded UP (the total may exceed the budget by less than one bit), where
+ * skim_oracle_allocate_bits rounds down to honour the "<=" of Section 4.2's constraint.
+ */
+int skim_oracle_allocate_bits_until(const float *err, int64_t rows, int n_bits, int b_min, double budget,
+                                    uint8_t *bits, int64_t *total)
+{
+    if (!err || !bits || rows <= 0 || n_bits <= 0 || b_min < 1) return -1;
+    int b_max = b_min + n_bits - 1;
+    if (!(budget >= (double)b_min && budget <= (double)b_max)) return -2;
+    double want = (double)rows * budget - 1e-6;
+    int64_t sum = rows * (int64_t)b_min;
+    for (int64_t i = 0; i < rows; ++i) bits[i] = (uint8_t)b_min;
+    while ((double)sum < want) {
+        int64_t best = -1;
+        double best_gain = 0.0;
+        for (int64_t i = 0; i < rows; ++i) {
+            if (bits[i] >= b_max) continue;
+            int b = bits[i] - b_min;
+            double gain = (double)err[i * n_bits + b] - (double)err[i * n_bits + b + 1];
+            if (best < 0 || gain > best_gain) { best = i; best_gain = gain; }
+        }
+        if (best < 0) break;
+        bits[best] += 1;
+        sum += 1;
+    }
+    if (total) *total = sum;
+    return 0;
+}
+
+/*
  * Allocation started from the floor of the budget (appendix with the results on other model
  * families: mixed precision is switched off at integer budgets, and at non-integer ones the
  * allocation is initialised with the budget rounded down).  Every row starts at floor(budget);

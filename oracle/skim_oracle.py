@@ -103,14 +103,18 @@ def cluster_rows(W, importance, bit_set, iters, s=None, row_bits=None, round_fp3
     return dict(centroids=centroids, codes=codes, err=err, trace=trace)
 
 
-def allocate_bits(err, b_min, budget, floor_start=False):
+def allocate_bits(err, b_min, budget, floor_start=False, round_up=False):
     """Greedy allocation over a float32 table [rows, n_bits]; returns (bits uint8 [rows], total).
-    floor_start: every row starts at floor(budget) instead of b_min."""
+    floor_start: every row starts at floor(budget) instead of b_min.  round_up: Algorithm 1's literal
+    stopping rule (until the total reaches rows * budget), i.e. the total rounded up."""
     err = np.ascontiguousarray(err, dtype=np.float32)
     rows, nb = err.shape
     bits = np.zeros(rows, dtype=np.uint8)
     total = C.c_int64(0)
     fn = lib().skim_oracle_allocate_bits_floor if floor_start else lib().skim_oracle_allocate_bits
+    if round_up:
+        assert not floor_start
+        fn = lib().skim_oracle_allocate_bits_until
     rc = fn(_p(err), C.c_int64(rows), C.c_int(nb), C.c_int(b_min), C.c_double(budget), _p(bits), C.byref(total))
     if rc == -2:
         raise ValueError("budget outside [b_min, b_max]")

@@ -204,6 +204,24 @@ int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int 
     return skim_launch_allocate(ctx, err, rows, bits, 0, K, bits_out);
 }
 
+int skim_allocate_bits_until(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
+                             double budget, uint8_t *bits_out, int64_t *total_bits)
+{
+    if (!ctx || !err || !bits_out) return SKIM_ERR_NULL;
+    SkimBits bits;
+    int rc = skim_check_bits(bit_set, n_bits, &bits);
+    if (rc) return rc;
+    if (rows < 1 || rows > 0x7fffffff) return SKIM_ERR_SHAPE;
+    if (!(budget >= (double)bits.b_min && budget <= (double)bits.b_max)) return SKIM_ERR_BUDGET;
+    int64_t T = (int64_t)ceil((double)rows * budget - 1e-6);      // the first total that is >= rows * budget
+    if (T < rows * (int64_t)bits.b_min) T = rows * (int64_t)bits.b_min;
+    if (T > rows * (int64_t)bits.b_max) T = rows * (int64_t)bits.b_max;
+    if (total_bits) *total_bits = T;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_allocate(ctx, err, rows, bits, 0, T - rows * (int64_t)bits.b_min, bits_out);
+}
+
 int skim_allocate_bits_floor(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits,
                              double budget, uint8_t *bits_out, int64_t *total_bits)
 {

@@ -20,7 +20,7 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
              -7: "SKIM_ERR_BAD_DATA", -8: "SKIM_ERR_SCALE", -9: "SKIM_ERR_ALIGN", -10: "SKIM_ERR_STATIC_LIMIT"}
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
-           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
+           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_bits_until", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
            "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
            "skim_kernel_times", "skim_strerror"]
@@ -168,15 +168,18 @@ class Skim:
                                         _ptr(cent), _ptr(codes), _ptr(err)), "skim_cluster_rows_at")
         return cent, codes, err
 
-    def allocate_bits(self, err, bit_set, budget, out=None, floor_start=False):
+    def allocate_bits(self, err, bit_set, budget, out=None, floor_start=False, round_up=False):
         """Returns (bits uint8 [rows], total_bits).  floor_start: every row starts at floor(budget)
-        instead of the smallest width (skim_allocate_bits_floor)."""
+        instead of the smallest width (skim_allocate_bits_floor).  round_up: the total is rounded up, Algorithm 1's
+        stopping rule as printed (skim_allocate_bits_until)."""
         _dev(err, torch.float32, "err")
         rows = err.shape[0]
         arr, nb, _ = _bits(bit_set)
         bits = out if out is not None else torch.empty((rows,), dtype=torch.uint8, device=err.device)
         total = C.c_int64()
         fn = lib().skim_allocate_bits_floor if floor_start else lib().skim_allocate_bits
+        if round_up:
+            fn = lib().skim_allocate_bits_until
         _chk(fn(self._h, _ptr(err), C.c_int64(rows), arr, C.c_int(nb), C.c_double(budget), _ptr(bits), C.byref(total)),
              "skim_allocate_bits_floor" if floor_start else "skim_allocate_bits")
         return bits, total.value

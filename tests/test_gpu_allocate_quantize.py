@@ -69,6 +69,17 @@ def test_floor_started_allocation_matches_oracle(ctx, oracle, rows):
             np.testing.assert_array_equal(got.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("rows", [1, 37, 1000, 5000])
+def test_allocation_with_the_printed_stopping_rule_matches_oracle(ctx, oracle, rows):
+    err = inputs.make_error_table(rows, 4, 900 + rows, monotone=False, ties=True)
+    errd = torch.from_numpy(err).cuda()
+    for budget in (1.0, 1.001, 2.25, 2.5003, 3.0, 3.9999, 4.0):
+        want, total = oracle.allocate_bits(err, 1, budget, round_up=True)
+        got, gtotal = ctx.allocate_bits(errd, BITS, budget, round_up=True)
+        assert gtotal == total
+        np.testing.assert_array_equal(got.cpu().numpy(), want, err_msg=f"rows={rows} budget={budget}")
+
+
 @pytest.mark.parametrize("rows", [1, 7, 300, 2000])
 def test_optimal_allocation_matches_oracle(ctx, oracle, rows):
     """skim_allocate_optimal: same recurrence, same order of additions, same tie rule as the oracle's dynamic

@@ -154,6 +154,24 @@ def test_optimal_allocation_equals_greedy_cost_when_gains_do_not_increase(oracle
         assert cost == sum(float(err[i, b - 1]) for i, b in enumerate(greedy))     # integers: exact
 
 
+def test_allocation_with_the_printed_stopping_rule(oracle):
+    """Algorithm 1 as printed stops once the total reaches rows * budget: restated here as a plain Python loop."""
+    rng = np.random.default_rng(11)
+    err = rng.integers(0, 60, size=(37, 4)).astype(np.float32)
+    for budget in (1.0, 1.01, 2.5, 3.2, 3.99, 4.0):
+        bits = [1] * 37
+        while sum(bits) < 37 * budget - 1e-6:
+            gains = [(float(err[i, b - 1]) - float(err[i, b]), -i) for i, b in enumerate(bits) if b < 4]
+            rows_left = [i for i, b in enumerate(bits) if b < 4]
+            best = max(range(len(gains)), key=lambda q: gains[q])
+            bits[rows_left[best]] += 1
+        got, total = oracle.allocate_bits(err, 1, budget, round_up=True)
+        assert list(got) == bits and total == sum(bits)
+        assert total == int(np.ceil(37 * budget - 1e-6))
+        down, tdown = oracle.allocate_bits(err, 1, budget)
+        assert tdown <= total <= tdown + 1
+
+
 # ---------------------------------------------------------------- emission
 
 def _unpack_row(words, cols, b):
