@@ -60,7 +60,7 @@ __device__ __forceinline__ int vec_slot(int j)
     return (j & ~(STEP - 1)) + (u >> 2) * 128 + lane * 4 + (u & 3);
 }
 
-constexpr int AHEAD = 8;            // steps whose words are fetched together, to have that many loads in flight
+constexpr int AHEAD = 4;            // steps whose words are fetched together; two such batches are in flight
 
 // The 8 codes of this lane in a step of B-bit codes, cut out of the step's 8B words (lane l < 8B holds
 // word l in `w`), as one word (code u in bits [u*B, (u+1)*B)).
@@ -83,12 +83,18 @@ __device__ __forceinline__ void unpack_row(const UnpackArgs &a, const float *vec
     __syncwarp();
     const int steps = (a.cols + STEP - 1) / STEP;
     float acc = 0.0f;
+    // the words of the next AHEAD steps are requested before the current ones are worked on
+    uint32_t wv[AHEAD], wn[AHEAD];
+#pragma unroll
+    for (int q = 0; q < AHEAD; ++q) {
+        const int w0 = q * 8 * B + lane;                       // lanes 0 .. 8B-1 fetch a step's words
+        wv[q] = (lane < 8 * B && w0 < stride) ? __ldg(words + w0) : 0u;
+    }
     for (int t0 = 0; t0 < steps; t0 += AHEAD) {
-        uint32_t wv[AHEAD];
 #pragma unroll
         for (int q = 0; q < AHEAD; ++q) {
-            const int w0 = (t0 + q) * 8 * B + lane;            // lanes 0 .. 8B-1 fetch a step's words
-            wv[q] = (lane < 8 * B && w0 < stride) ? __ldg(words + w0) : 0u;
+            const int w0 = (t0 + AHEAD + q) * 8 * B + lane;
+            wn[q] = (lane < 8 * B && w0 < stride) ? __ldg(words + w0) : 0u;
         }
 #pragma unroll
         for (int q = 0; q < AHEAD; ++q) {
@@ -123,6 +129,8 @@ __device__ __forceinline__ void unpack_row(const UnpackArgs &a, const float *vec
                 }
             }
         }
+#pragma unroll
+        for (int q = 0; q < AHEAD; ++q) wv[q] = wn[q];
     }
     if (MATVEC) {
 #pragma unroll
