@@ -86,7 +86,10 @@ int skim_max_cols(const skim_ctx *ctx, int64_t *out);
  * installed scale vector, so it must outlive every call that follows skim_apply_scale.  Most of
  * it is the clustering's scratch: about 13 bytes per element for min(rows, 8192) rows (the sorted
  * rows with their prefix sums, which the sort kernel hands to the Lloyd kernel); the scale update
- * adds 8 bytes x 296 x cols of partial gradients and 520 bytes per row. */
+ * adds 8 bytes x 296 x cols of partial gradients and 520 bytes per row.
+ * skim_set_workspace UNINSTALLS a scale vector that is installed (its reciprocal lives in the old
+ * workspace): call skim_apply_scale again afterwards.  The caller must not release the old workspace
+ * before the work already enqueued on the context's stream has finished. */
 int skim_workspace_bytes(int64_t rows, int64_t cols, size_t *out);
 int skim_set_workspace(skim_ctx *ctx, void *workspace, size_t bytes);
 
@@ -208,6 +211,8 @@ int skim_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, 
  *   - rows must not exceed SKIM_STATIC_MAX_ROWS, else SKIM_ERR_STATIC_LIMIT and nothing runs.
  *   - The first call on a device looks up the array's device address (one
  *     cudaGetSymbolAddress, cached per device); make that first call outside any stream capture.
+ *     The cached address does not survive cudaDeviceReset or the destruction of the device's
+ *     primary context: a process that does either must not call this function afterwards.
  *   - All calls on a device share the one array, and it keeps the previous call's contents
  *     (the call clears what it needs at zero).  Two calls that overlap on the GPU -- different
  *     streams, or different host threads -- race on it: serialise them.

@@ -178,10 +178,10 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
     if (tid == 0) { ps.misc[0] = 0; ps.misc[1] = 0; }
     __syncthreads();
     const SortedArrays<KeyT> src{skeys, sg};
-    const int nd = write_row_record<KeyT, THREADS, true>(a, src, ps, 0);
+    const int nd = write_row_record<KeyT, THREADS, true>(a, src, ps, 0, (int)blockIdx.x);
     if (nd <= 16) {
         collect_distinct<KeyT, THREADS>(src, m, nd, ps);
-        write_distinct_values(a, nd, ps.dvals);
+        write_distinct_values(a, nd, ps.dvals, (int)blockIdx.x);
     }
 }
 

@@ -300,7 +300,11 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         const bool landed = mbar_wait_bounded(mbar, 0);
         if (!__syncthreads_and(landed ? 1 : 0)) {
             // the copy never arrived: flag it, give it one more bounded chance to drain, leave
-            if (tid == 0) atomicOr(a.status, (unsigned long long)SKIM_STATUS_TIMEOUT);
+            // and mark the row record invalid, so that the Lloyd kernel skips the row
+            if (tid == 0) {
+                atomicOr(a.status, (unsigned long long)SKIM_STATUS_TIMEOUT);
+                *reinterpret_cast<int *>(a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride) = -1;
+            }
             mbar_wait_bounded(mbar, 0);
             return;
         }
@@ -320,10 +324,10 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         __syncthreads();
         nd = ps.misc[0];
     }
-    write_row_record<uint16_t, THREADS, false>(a, src, ps, nd);
+    write_row_record<uint16_t, THREADS, false>(a, src, ps, nd, (int)blockIdx.x);
     if (nd <= 16) {
         collect_distinct<uint16_t, THREADS>(src, m, nd, ps);
-        write_distinct_values(a, nd, ps.dvals);
+        write_distinct_values(a, nd, ps.dvals, (int)blockIdx.x);
     }
 }
 
@@ -331,13 +335,11 @@ struct Variant16 {
     int cap;
     int threads;
     void (*kernel)(ClusterArgs);
-    int dev_set;    // device on which the shared-memory attribute below was last set (-1: none)
-    int smem_set;
 };
 
-#define SKIM_V16(T, V) {T * V * 8, T, skim_sort16_kernel<T, V>, -1, 0}
+#define SKIM_V16(T, V) {T * V * 8, T, skim_sort16_kernel<T, V>}
 
-Variant16 kVariants[] = {
+const Variant16 kVariants[] = {
     SKIM_V16(128, 1), SKIM_V16(256, 1), SKIM_V16(512, 1), SKIM_V16(512, 2), SKIM_V16(512, 3), SKIM_V16(1024, 2),
     SKIM_V16(1024, 3),
 };
@@ -350,18 +352,15 @@ int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool laun
     // 128-bit loads of W rows and the bulk copy of importance rows need 16-byte aligned rows
     if ((reinterpret_cast<uintptr_t>(args.W) & 15u) || (args.ld % 8) != 0) return 1;
     if ((reinterpret_cast<uintptr_t>(args.G) & 15u) || (cols % 4) != 0) return 1;
-    for (Variant16 &v : kVariants) {
+    for (const Variant16 &v : kVariants) {
         if (v.cap < cols) continue;
         const Layout16 L = layout16((int)cols, v.threads);
         if (L.total > (size_t)ctx->max_smem_optin) continue;
         args.rec_stride = (long long)row_record(args.m).total;
         if (!launch) return SKIM_OK;
         const ClusterArgs a = args;
-        if (v.dev_set != ctx->device || v.smem_set != (int)L.total) {
-            SKIM_CUDA_OK(cudaFuncSetAttribute(v.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
-            v.dev_set = ctx->device;
-            v.smem_set = (int)L.total;
-        }
+        // set on every launch: a host-side call of microseconds, and no state shared between contexts
+        SKIM_CUDA_OK(cudaFuncSetAttribute(v.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total));
         v.kernel<<<(unsigned)rows, v.threads, L.total, ctx->stream>>>(a);
         SKIM_CUDA_OK(cudaGetLastError());
         ctx->launches += 1;

@@ -199,13 +199,14 @@ __device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, 
 // and returns the count; otherwise the caller passes the count (any number above 16 stands for
 // "more than 16") in nd_known.
 template <typename KeyT, int THREADS, bool COUNT, typename Src>
-__device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src &src, PhaseSmem &ps, int nd_known)
+__device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src &src, PhaseSmem &ps, int nd_known,
+                                                int local_row)
 {
     constexpr int NW = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int m = a.m;
     const RowRecord R = row_record(m);
-    unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
+    unsigned char *rec = a.scratch + (size_t)local_row * (size_t)a.rec_stride;     // local_row: the row's index inside the chunk
     float *gi = reinterpret_cast<float *>(rec + R.gi);
     int distinct = 0;
     unsigned bad = 0u;
@@ -267,7 +268,11 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
             if (lane >= off) { i0 += u0; i1 += u1; i2 += u2; }
         }
         if (lane == 31) { ps.segtot[sgm][0] = i0; ps.segtot[sgm][1] = i1; ps.segtot[sgm][2] = i2; }
-        double e0 = i0 - w0, e1 = i1 - w1, e2 = i2 - w2;     // sums from the segment start to the lane's first group
+        // sums from the segment start to the lane's first group: the neighbour's inclusive value itself,
+        // not inclusive minus own (which would add a rounding error of its own to every prefix)
+        double e0 = __shfl_up_sync(0xffffffffu, i0, 1), e1 = __shfl_up_sync(0xffffffffu, i1, 1),
+               e2 = __shfl_up_sync(0xffffffffu, i2, 1);
+        if (lane == 0) { e0 = 0.0; e1 = 0.0; e2 = 0.0; }
 #pragma unroll
         for (int h = 0; h < GPL; ++h) {
             const int q = q0 + h;
@@ -308,7 +313,9 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
             const double u2 = __shfl_up_sync(0xffffffffu, i2, off);
             if (lane >= off) { i0 += u0; i1 += u1; i2 += u2; }
         }
-        double b0 = i0 - run0, b1 = i1 - run1, b2 = i2 - run2;
+        double b0 = __shfl_up_sync(0xffffffffu, i0, 1), b1 = __shfl_up_sync(0xffffffffu, i1, 1),
+               b2 = __shfl_up_sync(0xffffffffu, i2, 1);
+        if (lane == 0) { b0 = 0.0; b1 = 0.0; b2 = 0.0; }
         double4 *seg = reinterpret_cast<double4 *>(rec + R.seg);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -322,9 +329,9 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
 }
 
 // Stores the row's distinct values (nd <= 16 of them, from collect_distinct) in the record header.
-__device__ __forceinline__ void write_distinct_values(const ClusterArgs &a, int nd, const float *dvals)
+__device__ __forceinline__ void write_distinct_values(const ClusterArgs &a, int nd, const float *dvals, int local_row)
 {
-    unsigned char *rec = a.scratch + (size_t)blockIdx.x * (size_t)a.rec_stride;
+    unsigned char *rec = a.scratch + (size_t)local_row * (size_t)a.rec_stride;
     if (threadIdx.x < 16) reinterpret_cast<float *>(rec + 64)[threadIdx.x] = threadIdx.x < nd ? dvals[threadIdx.x] : 0.0f;
 }
 

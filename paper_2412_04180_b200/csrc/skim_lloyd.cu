@@ -225,7 +225,10 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
             }
             break;
         }
-        if (normal && S0 > 0.0) c = (float)quotient(S1, S0);
+        // a cluster without weight keeps its centroid.  S0 is a difference of rounded prefix sums: over a
+        // run of zero importances that crosses a group or segment border it is rounding noise of either
+        // sign, not 0, so "has weight" means: above 2^-40 of the prefix it was taken from
+        if (normal && S0 > P0 * 0x1p-40) c = (float)quotient(S1, S0);
     }
     sm.errs[lane] = err_j;
     sm.tfs[lane] = has_boundary ? tf : INF;
@@ -274,7 +277,9 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
     LloydSmem &sm = sm_all[warp];
     const int64_t row = a.row0 + local;
     const unsigned char *rec = a.scratch + (size_t)local * (size_t)a.rec_stride;
-    const int nd = *reinterpret_cast<const int *>(rec);
+    const int nd_rec = *reinterpret_cast<const int *>(rec);
+    if (nd_rec < 0) return;                 // the sort kernel gave this row up (status word says why): no output
+    const int nd = max(nd_rec, 1);          // indexes sm.dvals below
     if (lane < 16) sm.dvals[lane] = reinterpret_cast<const float *>(rec + 64)[lane];
     // the row's group index, copied once
     const int nsk = sk_entries(a.m);
@@ -297,13 +302,8 @@ int skim_launch_lloyd(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
 {
     const unsigned blocks = (unsigned)((rows + LLOYD_WARPS - 1) / LLOYD_WARPS);
     const size_t smem = (size_t)LLOYD_WARPS * sk_entries(args.m) * sizeof(float);
-    static int attr_dev = -1;
-    static size_t attr_smem = 0;
-    if (attr_dev != ctx->device || attr_smem < smem) {
-        SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_dev = ctx->device;
-        attr_smem = smem;
-    }
+    // set on every launch: a host-side call of microseconds, and no state shared between contexts
+    SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     skim_lloyd_kernel<<<blocks, LLOYD_WARPS * 32, smem, ctx->stream>>>(args, (int)rows);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;

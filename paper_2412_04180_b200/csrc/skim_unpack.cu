@@ -177,16 +177,10 @@ __global__ void __launch_bounds__(UT) skim_unpack_kernel(UnpackArgs a)
 template <bool MATVEC>
 int launch_unpack(skim_ctx *ctx, const UnpackArgs &a)
 {
-    static int attr_dev[2] = {-1, -1};
-    static size_t attr_smem[2] = {0, 0};
     const size_t smem = (size_t)((a.cols + STEP - 1) / STEP * STEP) * sizeof(float);
     if (smem > (size_t)ctx->max_smem_optin) return SKIM_ERR_SHAPE;
-    const int f = MATVEC ? 1 : 0;
-    if (attr_dev[f] != ctx->device || attr_smem[f] < smem) {
-        SKIM_CUDA_OK(cudaFuncSetAttribute(skim_unpack_kernel<MATVEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_dev[f] = ctx->device;
-        attr_smem[f] = smem;
-    }
+    // set on every launch: a host-side call of microseconds, and no state shared between contexts
+    SKIM_CUDA_OK(cudaFuncSetAttribute(skim_unpack_kernel<MATVEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const unsigned blocks = (unsigned)(a.rows < ctx->sm_count ? a.rows : ctx->sm_count);   // one block per SM, rows dealt round-robin
     skim_unpack_kernel<MATVEC><<<blocks, UT, smem, ctx->stream>>>(a);
     SKIM_CUDA_OK(cudaGetLastError());

@@ -81,6 +81,7 @@ class Skim:
         _chk(lib().skim_create(C.byref(handle), C.c_int(device), sp), "skim_create")
         self._h = handle
         self._ws = None
+        self._scale = None      # the installed scale vector (kept so that a new workspace can take it over)
         if rows and cols:
             self.reserve(rows, cols)
 
@@ -108,25 +109,34 @@ class Skim:
         return out.value
 
     def reserve(self, rows, cols):
-        """Allocates (with torch) and installs a workspace big enough for rows x cols."""
+        """Allocates (with torch) and installs a workspace big enough for rows x cols.  A scale vector
+        that is installed moves to the new workspace with it."""
         nbytes = self.workspace_bytes(rows, cols)
         if self._ws is None or self._ws.numel() < nbytes:
-            self._ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
-            self.set_workspace(self._ws)
+            if self._ws is not None:
+                # work already enqueued on the context's stream may still use the old buffer
+                (self._stream.synchronize() if self._stream is not None else torch.cuda.synchronize(self.device))
+            self.set_workspace(torch.empty(nbytes, dtype=torch.uint8, device=self.device))
 
     def set_workspace(self, buf):
+        """Installs a caller-owned workspace.  skim_set_workspace drops an installed scale vector (its
+        reciprocal lives in the old workspace), so the binding installs it again in the new one."""
         _dev(buf, torch.uint8, "workspace")
         _chk(lib().skim_set_workspace(self._h, _ptr(buf), C.c_size_t(buf.numel())), "skim_set_workspace")
         self._ws = buf
+        if self._scale is not None:
+            self.apply_scale(self._scale)
 
     # ---- the path
     def apply_scale(self, s, cols=None):
         if s is None:
             _chk(lib().skim_apply_scale(self._h, C.c_void_p(0), C.c_int64(0)), "skim_apply_scale")
+            self._scale = None
             return
         _dev(s, torch.float32, "s")
         _chk(lib().skim_apply_scale(self._h, _ptr(s), C.c_int64(s.numel() if cols is None else cols)),
              "skim_apply_scale")
+        self._scale = s.clone() if cols is None else None     # a copy: callers update their vector in place
 
     def cluster_rows(self, W, importance, bit_set, iters, want_centroids=True, want_codes=False, ld=None,
                      cols=None):

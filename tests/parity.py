@@ -58,6 +58,37 @@ def check_cluster(ora, cent, err, codes, x_values, bit_set, rows=None, label="")
     return exact
 
 
+def check_cluster_at(ora, cent, err, codes, x_values, row_bits, bit_set, label=""):
+    """As check_cluster, for rows clustered only at their allocated width (skim_cluster_rows_at):
+    ora is oracle.cluster_rows(..., row_bits=row_bits); cent [rows, sumk], err [rows], codes [rows, cols]
+    from the GPU.  Centroids, error and labels of every row's own width block are compared."""
+    offs = offsets(bit_set)
+    bidx = {int(b): i for i, b in enumerate(bit_set)}
+    exact, total = 0, 0
+    for i, b in enumerate(row_bits):
+        b = int(b)
+        o, k, bi = offs[b], 1 << b, bidx[b]
+        oc = ora["centroids"][i, o:o + k]
+        gc = cent[i, o:o + k].astype(np.float64)
+        tol = CENT_RTOL * np.maximum(np.abs(oc), 1e-3 * np.abs(oc).max())
+        assert np.all(np.abs(gc - oc) <= tol), f"{label}: row {i} (width {b}) centroids differ: {gc} vs {oc}"
+        exact += int(np.sum(gc == oc))
+        total += k
+        if err is not None:
+            np.testing.assert_allclose(float(err[i]), ora["err"][i, bi], rtol=ERR_RTOL, atol=1e-30, err_msg=f"{label} row {i}")
+        if codes is not None:
+            want = ora["codes"][bi, i]
+            d = np.nonzero(codes[i] != want)[0]
+            assert len(d) <= (1.0 - LABEL_AGREE) * len(want) + 1, f"{label}: row {i}: {len(d)} labels differ"
+            for j in d:
+                lo, hi = sorted((int(codes[i, j]), int(want[j])))
+                assert hi == lo + 1, f"{label}: labels differ by more than one cluster"
+                x = x_values[i, j]
+                assert any(abs(x - 0.5 * (c[lo] + c[hi])) <= 4 * np.spacing(np.float32(abs(0.5 * (c[lo] + c[hi]))))
+                           for c in (gc, oc)), f"{label}: label mismatch away from a midpoint (row {i}, col {j})"
+    return exact / max(total, 1)
+
+
 def unpack_row(words, cols, b):
     bits = np.unpackbits(np.ascontiguousarray(words).view(np.uint8), bitorder="little")[:cols * b].reshape(cols, b)
     return (bits * (1 << np.arange(b))).sum(axis=1).astype(np.uint8)

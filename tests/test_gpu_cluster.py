@@ -134,6 +134,48 @@ def test_scaled_long_rows(ctx, oracle):
     check_cluster(ora, cent, err, codes, _values(w, s), BITS, label="scaled 22016")
 
 
+@pytest.mark.parametrize("cols", [8192, 11008, 16384])
+def test_scaled_rows_at_llama_lengths(ctx, oracle, cols):
+    """Scaled rows go through the 32-bit-key sort kernel; these three lengths take its three largest
+    variants below the 22 016-column one (8192 is the row length of the 22016 x 8192 matrix that
+    the scaling alternation runs on)."""
+    w, g = inputs.make_rows(24, cols, 8100 + cols, importance_sigma=2.0)
+    s = inputs.make_scale(cols, 29)
+    ora = oracle.cluster_rows(w, g, BITS, 50, s=s)
+    cent, err, codes = _gpu_cluster(ctx, w, g, BITS, 50, s=s)
+    exact = check_cluster(ora, cent, err, codes, _values(w, s), BITS, label=f"scaled cols={cols}")
+    assert exact > 0.98
+
+
+@pytest.mark.parametrize("cols", [12296, 14000, 16384, 16392, 20000])
+def test_unscaled_long_rows(ctx, oracle, cols):
+    """Row lengths between the LLaMA-7B and LLaMA-65B ones (each side of the limits at which the
+    fp16-key sort changes its kernel variant)."""
+    w, g = inputs.make_rows(12, cols, 8200 + cols)
+    ora = oracle.cluster_rows(w, g, BITS, 30)
+    cent, err, codes = _gpu_cluster(ctx, w, g, BITS, 30)
+    exact = check_cluster(ora, cent, err, codes, _values(w, None), BITS, label=f"cols={cols}")
+    assert exact > 0.98
+
+
+@pytest.mark.parametrize("cols,scaled", [(700, False), (11008, False), (3000, True)])
+def test_contiguous_run_of_zero_importance(ctx, oracle, cols, scaled):
+    """The largest 50 values of every row carry no importance at all, the rest spans many orders
+    of magnitude (exp(5 N)): the top clusters of the wide widths are weightless and must keep
+    their centroids, although their weight is a difference of two large rounded prefix sums."""
+    rows = 16
+    w, _ = inputs.make_rows(rows, cols, 8300 + cols)
+    rng = np.random.default_rng(cols)
+    g = np.exp(5.0 * rng.standard_normal((rows, cols))).astype(np.float32)
+    s = inputs.make_scale(cols, 31) if scaled else None
+    x = _values(w, s)
+    top = np.argsort(x, axis=1, kind="stable")[:, -50:]
+    np.put_along_axis(g, top, np.float32(0.0), axis=1)
+    ora = oracle.cluster_rows(w, g, BITS, 40, s=s)
+    cent, err, codes = _gpu_cluster(ctx, w, g, BITS, 40, s=s)
+    check_cluster(ora, cent, err, codes, x, BITS, label="zero-importance run")
+
+
 def test_cluster_rows_at_allocated_widths(ctx, oracle):
     rows, cols = 40, 1200
     w, g = inputs.make_rows(rows, cols, 123)

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from paper_2412_04180_b200 import inputs
-from parity import check_cluster, unpack_row
+from parity import check_cluster, check_cluster_at, unpack_row
 
 pytestmark = pytest.mark.gpu
 BITS = [1, 2, 3, 4]
@@ -158,53 +158,134 @@ def test_host_buffer_entry_point(ctx, oracle, skimlib):
     assert e.value.code == -5
 
 
-def _alternation_gpu(ctx, w, g, bits, rounds, steps, iters):
+def test_full_matrix_every_row(ctx, oracle):
+    """Every row of the benchmark's 4096 x 11008 matrix (the launch configuration the benchmark times):
+    centroids and errors of all four widths against the oracle, row by row.  A row whose
+    trajectory left the oracle's at a near-tie may end in another fixed point; such rows are counted,
+    capped at 0.1 % of the matrix, and must still be an equally good clustering."""
+    cfg = inputs.config(3)
+    rows, cols, seed = cfg["matrices"][1]
+    w, g = inputs.make_matrix(rows, cols, seed, importance_sigma=cfg["importance_sigma"])
+    cent, err, bits, total, out = _pipeline(ctx, w, g, cfg["iters"], 3.0)
+    ora = oracle.cluster_rows(w, g, BITS, cfg["iters"], want_codes=False)
+    oc, oe = ora["centroids"], ora["err"]
+    tol = 1e-4 * np.maximum(np.abs(oc), 1e-3 * np.abs(oc).max(axis=1, keepdims=True))
+    bad_c = (np.abs(cent.astype(np.float64) - oc) > tol).any(axis=1)
+    bad_e = (np.abs(err.astype(np.float64) - oe) > 1e-5 * np.abs(oe)).any(axis=1)
+    off_rows = np.nonzero(bad_c | bad_e)[0]
+    print(f"rows outside the tolerances: {len(off_rows)} of {rows}; "
+          f"centroids bit-identical: {np.mean(cent.astype(np.float64) == oc):.4f}")
+    assert len(off_rows) <= rows // 1000, off_rows[:20]
+    for i in off_rows:
+        np.testing.assert_allclose(err[i], oe[i], rtol=2e-3)      # another fixed point, as good as the oracle's
+    assert np.mean(cent.astype(np.float64) == oc) > 0.98
+    # downstream of the oracle's own table: the allocation and the packed form are bit-exact
+    _check_downstream_with_oracle_inputs(ctx, oracle, w, oe.astype(np.float32), oc.astype(np.float32), 3.0)
+
+
+def _row_labels(ora, bits):
+    return np.stack([ora["codes"][int(b) - 1, i] for i, b in enumerate(bits)]).astype(np.uint8)
+
+
+def _alternation_stagewise(ctx, oracle, w, g, bits, rounds, steps, iters, label):
+    """Algorithm 2 on the GPU, every stage of every round compared with the oracle on the SAME inputs.
+
+    Whole trajectories cannot be compared element-wise (the two alpha-updates differ in summation
+    order, and a 1e-9 change of alpha moves elements across cluster boundaries), but every stage can:
+    round r clusters W * (1/alpha_r) on both sides with the same binary32 alpha_r -- the vector the GPU
+    chain holds at that point, handed to the oracle as an input like any other scale vector --, and the
+    alpha-update is run on both sides from that alpha_r with the ORACLE's labels.  The GPU chain then
+    goes on from its own labels and its own alpha."""
     rows, cols = w.shape
     ctx.reserve(rows, cols)
     W, G, B = torch.from_numpy(w).cuda(), torch.from_numpy(g).cuda(), torch.from_numpy(bits).cuda()
     alpha = torch.ones(cols, device="cuda")
-    hist = []
-    for _ in range(rounds):
+    losses = []
+    for r in range(rounds):
+        a_r = alpha.cpu().numpy().copy()
         ctx.apply_scale(alpha)
         cent, codes, err = ctx.cluster_rows_at(W, G, B, BITS, iters)
-        trace = ctx.scale_update(W, G, codes, alpha, steps=steps)
-        hist.append((cent.cpu().numpy(), codes.cpu().numpy(), err.cpu().numpy(), trace.cpu().numpy(),
-                     alpha.cpu().numpy().copy()))
+        torch.cuda.synchronize()
+        assert ctx.get_status() == 0
+        ora = oracle.cluster_rows(w, g, BITS, iters, s=a_r, row_bits=bits)
+        x = (w.astype(np.float32) * (np.float32(1.0) / a_r)).astype(np.float64)
+        check_cluster_at(ora, cent.cpu().numpy(), err.cpu().numpy(), codes.cpu().numpy(), x, bits, BITS,
+                         label=f"{label} round {r + 1} clustering")
+        # the alpha-update of this round, both sides from alpha_r and the oracle's labels
+        olabels = _row_labels(ora, bits)
+        want_alpha, want_trace = oracle.scale_update(w, g, olabels, a_r.astype(np.float64), steps=steps)
+        a_t = torch.from_numpy(a_r.copy()).cuda()
+        trace_t = ctx.scale_update(W, G, torch.from_numpy(olabels).cuda(), a_t, steps=steps)
+        np.testing.assert_allclose(trace_t.cpu().numpy(), want_trace, rtol=1e-7, err_msg=f"{label} round {r + 1} loss trace")
+        np.testing.assert_allclose(a_t.cpu().numpy().astype(np.float64), want_alpha, rtol=1e-6,
+                                   err_msg=f"{label} round {r + 1} alpha")
+        # the GPU chain itself: its own labels, alpha updated in place
+        trace = ctx.scale_update(W, G, codes, alpha, steps=steps).cpu().numpy()
+        assert np.all(np.isfinite(trace))
+        # the update has no positivity constraint; a vector that reaches zero is outside the method's domain
+        assert float(alpha.min().item()) > 0.0, f"{label}: alpha left the positive range in round {r + 1}"
+        losses.append((trace[0], trace[-1]))
+    # final clustering and emission with the trained scale
+    a_f = alpha.cpu().numpy().copy()
     ctx.apply_scale(alpha)
     cent, codes, err = ctx.cluster_rows_at(W, G, B, BITS, iters)
     out = ctx.quantize(W, B, cent, BITS)
     torch.cuda.synchronize()
     assert ctx.get_status() == 0
     ctx.apply_scale(None)
-    return hist, cent.cpu().numpy(), codes.cpu().numpy(), {k: v.cpu().numpy() for k, v in out.items()}, alpha.cpu().numpy()
-
-
-def test_scaling_alternation_first_round_and_emission(ctx, oracle):
-    """Algorithm 2 with the allocated widths: round 1 is compared stage by stage with the oracle
-    (same inputs on both sides); later rounds cluster data that already differs in the last bits
-    of alpha, so they are checked through what must hold regardless: the loss trained by each
-    round goes down, and the final emission is bit-exact for the GPU's own alpha and centroids."""
-    rows, cols = 64, 768
-    w, g = inputs.make_rows(rows, cols, 5, importance_sigma=2.0)
-    bits = (np.arange(rows) % 4 + 1).astype(np.uint8)
-    hist, cent, codes, out, alpha = _alternation_gpu(ctx, w, g, bits, rounds=3, steps=30, iters=25)
-    # round 1: alpha = 1
-    ora = oracle.cluster_rows(w, g, BITS, 25, s=np.ones(cols, np.float32), row_bits=bits)
-    olabels = np.stack([ora["codes"][int(b) - 1, i] for i, b in enumerate(bits)])
-    assert np.mean(hist[0][1] == olabels) >= 0.999
-    want_alpha, want_trace = oracle.scale_update(w, g, olabels, np.ones(cols), steps=30)
-    if np.array_equal(hist[0][1], olabels):
-        np.testing.assert_allclose(hist[0][3], want_trace, rtol=1e-7)
-        np.testing.assert_allclose(hist[0][4].astype(np.float64), want_alpha, rtol=1e-6)
-    for h in hist:
-        assert h[3][-1] < h[3][0]
-    # emission with the trained scale: packed rows decode to the midpoint-count labels of the
-    # GPU's own centroids on the values W * (1/alpha) (numpy), and equal the labels it reported
-    _check_packed_rows(oracle, w, cent, bits, out, range(rows), s=alpha)
+    ora = oracle.cluster_rows(w, g, BITS, iters, s=a_f, row_bits=bits)
+    x = (w.astype(np.float32) * (np.float32(1.0) / a_f)).astype(np.float64)
+    check_cluster_at(ora, cent.cpu().numpy(), err.cpu().numpy(), codes.cpu().numpy(), x, bits, BITS,
+                     label=f"{label} final clustering")
+    # the packer is bit-exact when it is fed the oracle's centroids (same widths, same alpha)
+    oc32 = ora["centroids"].astype(np.float32)
+    ctx.apply_scale(torch.from_numpy(a_f).cuda())
+    out_o = ctx.quantize(W, B, torch.from_numpy(oc32).cuda(), BITS)
+    torch.cuda.synchronize()
+    ctx.apply_scale(None)
+    em = oracle.emit(w, bits, oc32, BITS, s=a_f)
+    words = int(out_o["group_info"][-1].item())
+    np.testing.assert_array_equal(out_o["packed"].cpu().numpy().view(np.uint32)[:words], em["packed"])
+    np.testing.assert_array_equal(out_o["row_order"].cpu().numpy(), em["row_order"])
+    np.testing.assert_array_equal(out_o["lut"].cpu().numpy().view(np.uint16), em["lut"])
+    # and the GPU chain's own packed rows decode to the labels it reported
+    out = {k: v.cpu().numpy() for k, v in out.items()}
+    codes = codes.cpu().numpy()
+    _check_packed_rows(oracle, w, cent.cpu().numpy(), bits, out, range(rows), s=a_f)
     pos_of = np.empty(rows, np.int64)
     pos_of[out["row_order"]] = np.arange(rows)
-    for i in range(0, rows, 7):
+    for i in range(0, rows, 3):
         b = int(bits[i])
         stride = oracle.row_stride_words(cols, b)
         start = out["group_info"][5 + b - 1] + (pos_of[i] - out["group_info"][b - 1]) * stride
         np.testing.assert_array_equal(unpack_row(out["packed"].view(np.uint32)[start:start + stride], cols, b), codes[i])
+    return losses
+
+
+def test_scaling_alternation_every_round(ctx, oracle):
+    """Algorithm 2 with the allocated widths on a small matrix: three rounds, every stage compared."""
+    rows, cols = 64, 768
+    w, g = inputs.make_rows(rows, cols, 5, importance_sigma=2.0)
+    bits = (np.arange(rows) % 4 + 1).astype(np.uint8)
+    losses = _alternation_stagewise(ctx, oracle, w, g, bits, rounds=3, steps=30, iters=25, label="64x768")
+    assert all(last < first for first, last in losses)       # 30 steps at the initial learning rate: every round's training lowers its loss
+
+
+@pytest.mark.parametrize("mat", [0, 1])
+def test_config5_schedule_on_a_row_subset(ctx, oracle, mat):
+    """The scaling alternation as the fifth configuration defines it -- five rounds of (re-clustering at the
+    allocated widths for 50 Lloyd iterations, then 120 Adam steps on alpha with the learning rate halved
+    every 40) -- on a row subset of both LLaMA-65B shapes, with the widths of a 3.0-bit allocation."""
+    cfg = inputs.config(5)
+    rows_total, cols, seed = cfg["matrices"][mat]
+    # few rows per column let alpha over-fit its columns; the 22 016-column shape needs more rows than the
+    # 8192-column one for every entry to stay positive through all five rounds
+    nrows = 16 if mat == 0 else 64
+    w, g = inputs.make_rows(rows_total, cols, seed, 1024, nrows, importance_sigma=cfg["importance_sigma"])
+    table = oracle.cluster_rows(w, g, BITS, cfg["iters"], want_codes=False)["err"].astype(np.float32)
+    bits, total = oracle.allocate_bits(table, 1, 3.0)
+    assert total == 3 * nrows
+    losses = _alternation_stagewise(ctx, oracle, w, g, bits, rounds=cfg["scale_rounds"], steps=120, iters=cfg["iters"],
+                                    label=f"config5/{mat}")
+    assert len(losses) == 5
+
