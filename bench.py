@@ -42,6 +42,7 @@ CLUSTER_BYTES_PER_ROW = 136
 # (bytes), or None when the kernel changed since the counters were taken.
 SORT_TRAFFIC_BYTES_PER_ROW = 179_290   # (135.38 MB read + 231.80 MB written) / 2048 rows, profiles/skim_sort16_kernel_2048x11008.md
 DOMINANT_KERNEL = "skim_sort16_kernel"
+DTYPE = "f64 sums, f32 centroid state (fp16 weights and fp32 importance in)"
 
 
 def measured_peak():
@@ -142,8 +143,8 @@ def run_reference(args):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "rows/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample_rows_per_step": nrows},
+        "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+        "config": {"workload": WORKLOAD, "rows": ROWS, "cols": COLS, "sample_rows_per_step": nrows},
         "cpu_baseline": {"value": value, "unit": "rows/s", "cores": orc.num_threads(), "kind": "oracle",
                          "sample": f"first {nrows} of {ROWS} rows of the same matrix per step, full pipeline"},
         "e2e": {"value": value, "unit": "rows/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -282,6 +283,7 @@ def run_ours(args):
     sort_total, lloyd_total, timed_chunks = ctx.kernel_times()
     ctx.kernel_timing(False)
     sort_ms, lloyd_ms = sort_total / max(1, timed_chunks), lloyd_total / max(1, timed_chunks)
+    iter_sum, iter_rows = ctx.lloyd_iterations()
     busy(0.4)
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
@@ -295,6 +297,62 @@ def run_ours(args):
     total_bits = int(bits.sum().item())
     assert total_bits == int(ROWS * BUDGET), total_bits
     mx = Skim.packed_layout(ROWS, COLS, BIT_SET)[1]
+
+    # the same step with the converged-row shortcut off: every row runs all ITERS iterations (same output)
+    extra = {}
+    if not args.rows:
+        ctx.early_exit(False)
+        for _ in range(3):
+            step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        stream.synchronize()
+        ctx.early_exit(True)
+        extra["ms_per_step_early_exit_off"] = e0.elapsed_time(e1) / args.steps
+
+        # Algorithm 2 on the same matrix at the allocated widths (outside the timed region): the alpha-update
+        # alone, and one whole alternation round = re-clustering at b_i + 120 Adam steps + emission
+        peak_s, _ = measured_peak()
+        with torch.cuda.stream(stream):
+            alpha = torch.ones(COLS, dtype=torch.float32, device="cuda")
+            ctx.apply_scale(alpha)
+            cent_at = cent.clone()
+            _, labels, _ = ctx.cluster_rows_at(W, G, bits, BIT_SET, ITERS, want_codes=True, centroids=cent_at)
+            ctx.scale_update(W, G, labels, alpha, steps=3, want_trace=False)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            ctx.scale_update(W, G, labels, alpha, steps=40, want_trace=False)
+            e1.record(stream)
+            stream.synchronize()
+            adam_ms = e0.elapsed_time(e1) / 40
+            adam_bytes = 2 * 7 * ROWS * COLS          # two passes over fp16 W, fp32 importance and u8 labels
+            r0, r1, r2, r3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+            r0.record(stream)
+            ctx.apply_scale(alpha)
+            _, labels, _ = ctx.cluster_rows_at(W, G, bits, BIT_SET, ITERS, want_codes=True, centroids=cent_at)
+            r1.record(stream)
+            ctx.scale_update(W, G, labels, alpha, steps=120, want_trace=False)
+            r2.record(stream)
+            ctx.apply_scale(alpha)
+            ctx.quantize(W, bits, cent_at, BIT_SET, out=out)
+            r3.record(stream)
+            stream.synchronize()
+            ctx.apply_scale(None)
+            assert ctx.get_status() == 0
+        extra["scale_update"] = {"ms_per_adam_step": adam_ms, "algorithmic_bytes_per_step": adam_bytes,
+                                 "hbm_frac": adam_bytes / (adam_ms * 1e-3) / 1e9 / peak_s, "kernels_per_step": 3}
+        extra["alternation_round"] = {"recluster_at_allocated_widths_ms": r0.elapsed_time(r1),
+                                      "adam_120_steps_ms": r1.elapsed_time(r2), "emit_ms": r2.elapsed_time(r3),
+                                      "total_ms": r0.elapsed_time(r3),
+                                      "note": "one round of Algorithm 2 on the same matrix with the scale vector installed "
+                                              "(32-bit keys), labels written; single measurement, outside the timed region"}
+        # the pipeline's own outputs again (the round above overwrote the packed form with the scaled one)
+        step()
+        stream.synchronize()
 
     # the consumers of the packed form (outside the timed region; reported beside the step)
     consumers = None
@@ -370,16 +428,20 @@ def run_ours(args):
     result = {
         "metric": METRIC, "value": job_rows_per_s, "unit": "rows/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": WORKLOAD, "rows": ROWS, "cols": COLS, "l2": "inputs 270 MB per step exceed the 126 MB L2",
-                   "early_exit": "on (bit-identical)", "parallelism": f"{world} independent matrices"},
+                   "early_exit": "on (rows stop once no boundary moved; output bit-identical to running all iterations)",
+                   "parallelism": f"{world} independent matrices"},
+        "lloyd_iterations_mean": (iter_sum / iter_rows) if iter_rows else None, "lloyd_iterations_max": ITERS,
         "weights_per_s": world * ROWS * COLS / (ms_step / 1e3),
         "stage_ms": {"cluster": cluster_ms, "allocate": alloc_ms, "quantize": quant_ms},
         "kernel_ms": {"skim_sort16_kernel": sort_ms, "skim_lloyd_kernel": lloyd_ms, "launches_timed": timed_chunks},
         "pipeline_hbm_frac": pipeline_bytes / (ms_step * 1e-3) / 1e9 / peak,
         "cluster_stage_hbm_frac": cluster_bytes / (cluster_ms * 1e-3) / 1e9 / peak,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "consumers": consumers,
-        "roofline": {"bound": "hbm", "kernel": DOMINANT_KERNEL, "achieved": achieved, "peak": peak,
+        **extra,
+        "roofline": {"bound": "hbm", "limiter": "shared-memory wavefronts and instruction issue (ncu); HBM is the roofline the target names",
+                     "kernel": DOMINANT_KERNEL, "achieved": achieved, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "traffic": SORT_TRAFFIC_BYTES_PER_ROW * ROWS if SORT_TRAFFIC_BYTES_PER_ROW else None,
                      "algorithmic_bytes": sort_bytes, "kernel_ms": sort_ms},

@@ -70,6 +70,7 @@ extern "C" {
 #define SKIM_STATUS_BAD_SCALE 4ull       /* zero, negative or non-finite scale entry */
 #define SKIM_STATUS_BAD_BITS 8ull        /* an allocated width that is not in bit_set (row skipped) */
 #define SKIM_STATUS_TIMEOUT 16ull        /* an asynchronous copy did not complete within its wait limit (row skipped) */
+#define SKIM_STATUS_BOUNDS 32ull         /* checked build only (-DSKIM_CHECK_BOUNDS): a computed index was out of range (access skipped) */
 
 typedef struct skim_ctx skim_ctx;
 
@@ -301,6 +302,19 @@ int64_t skim_launch_count(const skim_ctx *ctx);
  */
 int skim_kernel_timing(skim_ctx *ctx, int enable);
 int skim_kernel_times(skim_ctx *ctx, double *sort_ms, double *lloyd_ms, int64_t *chunks);
+
+/*
+ * Measurement aids for the iteration count (no counterpart in the paper, which states no stopping
+ * rule).  The clustering runs exactly `iters` assign/update pairs per row, except that a row stops as
+ * soon as an assignment moved no boundary: every later pair would reproduce the same state bit for
+ * bit, so the result is the same.  skim_early_exit(ctx, 0) switches that shortcut off (all rows run
+ * all `iters` pairs; same output, more time), skim_early_exit(ctx, 1) restores the default.
+ * While skim_kernel_timing is enabled the Lloyd kernel also adds up the pairs each row really ran;
+ * skim_lloyd_iterations reads and clears that count (it waits for the stream): `iterations` = pairs
+ * summed over rows, `rows` = rows counted (host pointers, either may be NULL).
+ */
+int skim_early_exit(skim_ctx *ctx, int enable);
+int skim_lloyd_iterations(skim_ctx *ctx, int64_t *iterations, int64_t *rows);
 
 const char *skim_strerror(int code);
 

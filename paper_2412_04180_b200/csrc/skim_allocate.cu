@@ -132,7 +132,10 @@ __global__ void __launch_bounds__(AT) skim_allocate_kernel(const float *__restri
                 live[t] = row_ok && t < steps && (pass == 0 || (key >> (shift + 8)) == prefix);
                 dig[t] = live[t] ? (unsigned)((key >> shift) & 0xffull) : 0u;
                 if (live[t] && first < 0) first = t;
-                if (collect && live[t]) list[atomicAdd(&s_count, 1u)] = key;
+                if (collect && live[t]) {
+                    const unsigned slot = atomicAdd(&s_count, 1u);
+                    if (SKIM_IDX(slot, LIST_CAP, nullptr)) list[slot] = key;
+                }
             }
             if (!have_digit) {
                 const unsigned any = __ballot_sync(0xffffffffu, first >= 0);

@@ -74,6 +74,7 @@ int skim_create(skim_ctx **out, int device, void *cuda_stream)
     ctx->scale_cols = 0;
     ctx->launches = 0;
     ctx->copy_ready = false;
+    ctx->early_exit = true;
     ctx->timing = false;
     ctx->timing_ready = false;
     ctx->timing_used = 0;
@@ -536,6 +537,29 @@ int skim_kernel_times(skim_ctx *ctx, double *sort_ms, double *lloyd_ms, int64_t 
     if (sort_ms) *sort_ms = s;
     if (lloyd_ms) *lloyd_ms = l;
     if (chunks) *chunks = ctx->timing_used;
+    return SKIM_OK;
+}
+
+int skim_early_exit(skim_ctx *ctx, int enable)
+{
+    if (!ctx) return SKIM_ERR_NULL;
+    ctx->early_exit = enable != 0;
+    return SKIM_OK;
+}
+
+int skim_lloyd_iterations(skim_ctx *ctx, int64_t *iterations, int64_t *rows)
+{
+    if (!ctx) return SKIM_ERR_NULL;
+    if (!ctx->ws) return SKIM_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    unsigned long long v[2] = {0ull, 0ull};
+    unsigned char *p = (unsigned char *)ctx->ws + 8;
+    SKIM_CUDA_OK(cudaMemcpyAsync(v, p, 16, cudaMemcpyDeviceToHost, ctx->stream));
+    SKIM_CUDA_OK(cudaMemsetAsync(p, 0, 16, ctx->stream));
+    SKIM_CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    if (iterations) *iterations = (int64_t)v[0];
+    if (rows) *rows = (int64_t)v[1];
     return SKIM_OK;
 }
 

@@ -159,8 +159,10 @@ __global__ void __launch_bounds__(THREADS) skim_sort_kernel(ClusterArgs a)
             if (rank == 0) cnt[warp * RADIX + d] = base + __popc(peers);
             __syncwarp();
             const uint32_t pos = dbase[d] + base + rank;
-            skeys[pos] = key[i];
-            sg[pos] = val[i];
+            if (SKIM_IDX(pos, CAP, a.status)) {
+                skeys[pos] = key[i];
+                sg[pos] = val[i];
+            }
         }
         __syncthreads();
         if (pass + 1 < PASSES) {
@@ -256,6 +258,8 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     a.scratch = ws.cluster_scratch;
     a.rec_stride = 0;
     a.row0 = 0;
+    a.early_exit = ctx->early_exit ? 1 : 0;
+    a.iter_stats = ctx->timing ? ws.status + 1 : nullptr;
 
     // plan: the fp16-key sort kernel when it applies, else the generic one
     bool fast = !scaled && skim_launch_sort16(ctx, a, 0, false) == SKIM_OK;

@@ -104,6 +104,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
 struct SortedItems16 {
     const uint32_t *items;
     const float *graw;
+    unsigned long long *status;
     __device__ __forceinline__ unsigned group(int e, int m, uint16_t *ks, float *gs) const
     {
         const uint4 a = *reinterpret_cast<const uint4 *>(items + e), b = *reinterpret_cast<const uint4 *>(items + e + 4);
@@ -112,7 +113,7 @@ struct SortedItems16 {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             ks[u] = (uint16_t)(it[u] >> 16);
-            const float g = (e + u < m) ? graw[it[u] & 0xffffu] : 0.0f;
+            const float g = (e + u < m && SKIM_IDX(it[u] & 0xffffu, m, status)) ? graw[it[u] & 0xffffu] : 0.0f;
             bits |= __float_as_uint(g);
             gs[u] = g;
         }
@@ -221,10 +222,11 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
             const uint32_t key = item[i] >> 16;
             const uint32_t pos = C0[key & (D0 - 1)] + (item[i] & 0xffffu);      // bin base + slot
             const uint32_t col = (uint32_t)(((i >> 3) * THREADS + tid) * 8 + (i & 7));
-            buf[pos] = (key << 16) | col;
+            if (SKIM_IDX(pos, m, a.status)) buf[pos] = (key << 16) | col;
             // one more item of digit key >> 12 in the stretch of pass-1 owner pos / ITEMS
             const uint32_t owner = pos / ITEMS;
-            atomicAdd(&cnt1w[((key >> D0_BITS) * THREADS + owner) >> 1], (owner & 1u) ? 0x10000u : 1u);
+            if (SKIM_IDX(owner, THREADS, a.status))
+                atomicAdd(&cnt1w[((key >> D0_BITS) * THREADS + owner) >> 1], (owner & 1u) ? 0x10000u : 1u);
         }
     }
     // the pass-0 counters are dead: their place takes the importance row, by the asynchronous proxy
@@ -290,7 +292,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
             uint16_t *c = cnt1 + (item[i] >> (16 + D0_BITS)) * THREADS + tid;
             const uint32_t pos = *c;
             *c = (uint16_t)(pos + 1u);
-            buf[pos] = item[i];
+            if (SKIM_IDX(pos, m, a.status)) buf[pos] = item[i];
         }
     }
 
@@ -310,7 +312,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         }
     }
     // ---------------------------------------------------------------- row record
-    const SortedItems16 src{buf, graw};
+    const SortedItems16 src{buf, graw, a.status};
     int nd = ps.misc[0];                     // more than 16 occupied bins: more than 16 distinct values
     if (nd <= 16) {
         // few bins: count the distinct values themselves

@@ -81,6 +81,8 @@ struct ClusterArgs {
     unsigned char *scratch;   // row records of the current chunk (written by the sort kernel, read by the Lloyd kernel)
     long long rec_stride;     // bytes between row records
     int64_t row0;             // first row of the current chunk
+    int early_exit;           // stop a row once no boundary moved
+    unsigned long long *iter_stats;   // nullptr, or two counters: iterations run, rows counted
 };
 
 // Row record: what the sort kernel leaves in global memory for the Lloyd kernel.  All offsets are
@@ -174,7 +176,7 @@ __device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, 
     for (int p = threadIdx.x; p < m; p += THREADS) {
         if (p == 0 || src.key_at(p) != src.key_at(p - 1)) {
             const int slot = atomicAdd(&ps.misc[1], 1);
-            if (slot < 16) ps.tfs[slot] = __int_as_float(p);
+            if (slot >= 0 && slot < 16) ps.tfs[slot] = __int_as_float(p);
         }
     }
     __syncthreads();
@@ -184,7 +186,7 @@ __device__ __forceinline__ void collect_distinct(const Src &src, int m, int nd, 
         int rank = 0;
         for (int u = 0; u < nd; ++u) rank += (__shfl_sync(0xffffffffu, p, u) < p) ? 1 : 0;
         __syncwarp();
-        if (lane < nd) ps.dvals[rank] = KeyOps<KeyT>::to_float(src.key_at(p));
+        if (lane < nd && SKIM_IDX(rank, 32, nullptr) && SKIM_IDX(p, m, nullptr)) ps.dvals[rank] = KeyOps<KeyT>::to_float(src.key_at(p));
     }
     __syncthreads();
 }
@@ -267,7 +269,7 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
             const double u2 = __shfl_up_sync(0xffffffffu, i2, off);
             if (lane >= off) { i0 += u0; i1 += u1; i2 += u2; }
         }
-        if (lane == 31) { ps.segtot[sgm][0] = i0; ps.segtot[sgm][1] = i1; ps.segtot[sgm][2] = i2; }
+        if (lane == 31 && SKIM_IDX(sgm, 96, a.status)) { ps.segtot[sgm][0] = i0; ps.segtot[sgm][1] = i1; ps.segtot[sgm][2] = i2; }
         // sums from the segment start to the lane's first group: the neighbour's inclusive value itself,
         // not inclusive minus own (which would add a rounding error of its own to every prefix)
         double e0 = __shfl_up_sync(0xffffffffu, i0, 1), e1 = __shfl_up_sync(0xffffffffu, i1, 1),

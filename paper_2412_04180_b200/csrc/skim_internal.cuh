@@ -30,6 +30,7 @@ struct skim_ctx {
     bool copy_ready;
     // optional kernel timing: events before the sort kernel, between the two kernels and after
     // the Lloyd kernel of every clustering chunk, on the context's stream
+    bool early_exit;      // rows stop iterating once no boundary moved (default)
     bool timing;
     bool timing_ready;
     int timing_used;
@@ -39,7 +40,7 @@ struct skim_ctx {
 // Workspace layout (all offsets 256-byte aligned), carved per call for the call's (rows, cols).
 // The status word and the reciprocal scale sit at fixed offsets, so they persist across calls.
 struct SkimWorkspace {
-    unsigned long long *status;  // 1 word
+    unsigned long long *status;  // word 0: status bits; words 1, 2: Lloyd iterations run and rows counted (skim_lloyd_iterations)
     float *rscale;               // [cols]     reciprocal of the installed scale vector
     int32_t *row_pos;            // [rows]     packed-row index of every source row
     double *alpha64;             // [cols]     scale-update master copy of alpha
@@ -87,6 +88,23 @@ static inline SkimWorkspace skim_carve(void *base, int64_t rows, int64_t cols)
     w.bytes = off;
     return w;
 }
+
+// Index checks of the checked build (nvcc -DSKIM_CHECK_BOUNDS; build.py builds it as libskim_checked.so).
+// Every index into shared memory, a row record or a scratch list that is COMPUTED from data (a scatter
+// position, a counter slot, a searched group, a gathered column) goes through SKIM_IDX: in the checked
+// build an index outside [0, n) sets SKIM_STATUS_BOUNDS in the status word and the access is skipped
+// (never a trap); in the normal build the macro is the constant true and costs nothing.
+#ifdef SKIM_CHECK_BOUNDS
+__device__ __forceinline__ bool skim_index_ok(long long i, long long n, unsigned long long *status)
+{
+    if (i >= 0 && i < n) return true;
+    if (status) atomicOr(status, (unsigned long long)SKIM_STATUS_BOUNDS);
+    return false;
+}
+#define SKIM_IDX(i, n, status) skim_index_ok((long long)(i), (long long)(n), (status))
+#else
+#define SKIM_IDX(i, n, status) true
+#endif
 
 // Validated description of a bit set.
 struct SkimBits {

@@ -79,7 +79,7 @@ struct Window {
     int ws;
     __device__ __forceinline__ void load(const float *gi, int ngi, int guess)   // gi: shared memory
     {
-        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, ngi - WIN));
+        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, ngi - WIN));     // may reach into the 16 padding entries behind the index
         const float4 *p = reinterpret_cast<const float4 *>(gi + ws);
 #pragma unroll
         for (int q = 0; q < 4; ++q) v[q] = p[q];
@@ -148,7 +148,8 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
     if (degenerate) c = sm.dvals[min(j, nd - 1)];
     if (normal) {
         const int idx = (int)(((long long)(2 * j + 1) * m) / (2 * k));
-        c = __ldg(reinterpret_cast<const float *>(groups + (size_t)(idx >> 3) * SKIM_GROUP_BYTES) + (idx & 7));
+        if (SKIM_IDX(idx, m, a.status))
+            c = __ldg(reinterpret_cast<const float *>(groups + (size_t)(idx >> 3) * SKIM_GROUP_BYTES) + (idx & 7));
     }
 
     int Bprev = -1;
@@ -183,6 +184,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 nle = lo;
             }
             grp_i = max(nle - 1, 0);
+            if (!SKIM_IDX(grp_i, R.ngrp, a.status)) grp_i = 0;
             gstep = gprev >= 0 ? grp_i - gprev : 0;
             gprev = grp_i;
             const unsigned char *gr = groups + (size_t)grp_i * SKIM_GROUP_BYTES;
@@ -191,7 +193,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
             B = min((grp_i << 3) + cntk, m);
         }
         const bool same = __all_sync(0xffffffffu, B == Bprev);
-        const bool final = (it >= a.iters) || same;
+        const bool final = (it >= a.iters) || (same && a.early_exit);
         Bprev = B;
         double P0 = 0.0, P1 = 0.0, Pc = 0.0;
         if (normal) {
@@ -222,6 +224,10 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
             if (normal) {
                 const double cd = (double)c, S2 = Pc - Qc;
                 err_j = fmax(fma(cd, fma(cd, S0, -2.0 * S1), S2), 0.0);
+            }
+            if (a.iter_stats && lane == 0) {
+                atomicAdd(a.iter_stats, (unsigned long long)it);       // assign/update pairs this row ran
+                atomicAdd(a.iter_stats + 1, 1ull);
             }
             break;
         }

@@ -48,6 +48,7 @@ __device__ __forceinline__ bool locate_row(const UnpackArgs &a, int64_t p, int &
     stride = (int)skim_row_stride_words(a.cols, width);
     words = a.packed + a.group_info[a.nb + 1 + bi] + (p - a.group_info[bi]) * (int64_t)stride;
     src_row = a.row_order[p];
+    if (!SKIM_IDX(src_row, a.rows, nullptr)) return false;
     return true;
 }
 

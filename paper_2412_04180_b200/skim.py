@@ -12,7 +12,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libskim.so")
+# SKIM_LIB selects another build of the same library (the bounds-checked one, build.py --checked)
+LIB_PATH = os.environ.get("SKIM_LIB") or os.path.join(_HERE, "libskim.so")
 _lib = None
 
 ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_ERR_BITSET",
@@ -23,7 +24,7 @@ EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes
            "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_bits_until", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
            "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
-           "skim_kernel_times", "skim_strerror"]
+           "skim_kernel_times", "skim_early_exit", "skim_lloyd_iterations", "skim_strerror"]
 
 
 class SkimError(RuntimeError):
@@ -321,6 +322,17 @@ class Skim:
         s, l, n = C.c_double(), C.c_double(), C.c_int64()
         _chk(lib().skim_kernel_times(self._h, C.byref(s), C.byref(l), C.byref(n)), "skim_kernel_times")
         return s.value, l.value, n.value
+
+
+    def early_exit(self, enable=True):
+        """Measurement aid: rows stop iterating once no boundary moved (default) or always run all iterations."""
+        _chk(lib().skim_early_exit(self._h, C.c_int(1 if enable else 0)), "skim_early_exit")
+
+    def lloyd_iterations(self):
+        """Returns (iterations summed over rows, rows counted) since the last call, while kernel_timing is on."""
+        it, n = C.c_int64(), C.c_int64()
+        _chk(lib().skim_lloyd_iterations(self._h, C.byref(it), C.byref(n)), "skim_lloyd_iterations")
+        return it.value, n.value
 
 
 STATIC_MAX_ROWS = 65536

@@ -241,3 +241,49 @@ def test_argument_errors(ctx, skimlib):
     assert e.value.code == -8
     ctx.apply_scale(None)
     assert ctx.max_cols() >= 22016
+
+
+def test_bounds_checked_build_reports_no_violation(skimlib):
+    """The checked build (every computed index into shared memory, a row record or a scratch list is
+    range-checked; a violation sets a status bit and skips the access) runs the ragged column counts, the
+    degenerate rows, the long rows and a scaled case, in a process of its own, with a clean status word:
+    the tests it runs assert status == 0 after every clustering call."""
+    import os
+    import subprocess
+    import sys
+    from paper_2412_04180_b200 import build
+    lib = build.build(checked=True)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SKIM_LIB=lib)
+    cmd = [sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_cluster.py"), "-q", "-x", "-m", "gpu",
+           "-k", "ragged_column_counts or degenerate_rows or unscaled_long_rows or test_scaled_rows or zero_importance",
+           "-p", "no:cacheprovider"]
+    res = subprocess.run(cmd, cwd=root, env=env, capture_output=True, text=True, timeout=1200)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+    assert " passed" in res.stdout and "failed" not in res.stdout
+
+
+def test_early_exit_switch_and_iteration_count(ctx):
+    """With the converged-row shortcut off every row runs all iterations; the output is bit-identical
+    (a row whose boundaries stopped moving reproduces its state), and the iteration counter says so."""
+    rows, cols, iters = 40, 2048, 60
+    w, g = inputs.make_rows(rows, cols, 77)
+    w[3, :] = np.float16(0.5)                    # a degenerate row: no iteration changes anything
+    W, G = torch.from_numpy(w).cuda(), torch.from_numpy(g).cuda()
+    ctx.reserve(rows, cols)
+    ctx.apply_scale(None)
+    ctx.kernel_timing(True)
+    cent1, _, err1 = ctx.cluster_rows(W, G, BITS, iters)
+    it_on, n_on = ctx.lloyd_iterations()
+    ctx.early_exit(False)
+    cent0, _, err0 = ctx.cluster_rows(W, G, BITS, iters)
+    it_off, n_off = ctx.lloyd_iterations()
+    ctx.early_exit(True)
+    ctx.kernel_timing(False)
+    torch.cuda.synchronize()
+    assert torch.equal(cent0, cent1) and torch.equal(err0, err1)
+    assert n_on == rows and n_off == rows
+    assert it_off == rows * iters
+    assert 0 < it_on <= it_off
+    ctx.cluster_rows(W, G, BITS, iters)
+    assert ctx.lloyd_iterations() == (0, 0)      # nothing is counted while timing is off

