@@ -16,6 +16,7 @@
  *   - packing rows grouped by bit-width                   -- Section 4.2, last paragraph.
  *   - unpacking: dequantised weights and the matrix-vector product from the packed form
  *                                                         -- Section 4 overview, Sections 4.2, 4.3.
+ *   - the L-full error  (w - wq) X X^T (w - wq)^T  of a row -- Section 3.4; Section 4.2; Algorithm 3.
  *
  * Readings where the paper is silent (kept identical on the CUDA side):
  *   - init: centroid j of k = sorted_row[ floor((2j+1) m / (2k)) ] (index quantiles).
@@ -678,6 +679,82 @@ int skim_oracle_scale_update(const uint16_t *W, const float *importance, int64_t
     }
     free(m1); free(m2); free(grad);
     return rc;
+}
+
+/* ------------------------------------------------------------------ L-full error (Section 3.4) */
+
+/*
+ * Residual of a row against its quantised form, the operand of the L-full error (Section 3.4: the error of
+ * row i is (w_i - wq_i) X X^T (w_i - wq_i)^T; Section 4 overview and Section 4.3: wq = replace(c, l) * alpha).
+ *   label   the 1-D quantiser rule on the clustered value (as in skim_oracle_emit)
+ *   wq      the binary32 product  c[label] * alpha_j   (alpha == NULL: c[label] itself)
+ *   d       binary16( (float(w) - wq) * 2^exp2 ), the difference taken in binary32, the power-of-two scaling
+ *           exact, then one rounding to nearest even.  The scaling keeps small residuals out of the
+ *           binary16 subnormal range; the error routine divides it out again.
+ * row_bits == NULL: every row uses the centroid block of `width`; else row i uses width row_bits[i].
+ * D out [rows][ldd] binary16 bit patterns.
+ */
+int skim_oracle_residual(const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *s,
+                         const uint8_t *row_bits, int width, const float *centroids, const int *bit_set,
+                         int n_bits, int exp2, uint16_t *D, int64_t ldd)
+{
+    if (!W || !centroids || !D || rows <= 0 || cols <= 0 || ld < cols || ldd < cols) return -1;
+    if (check_bit_set(bit_set, n_bits)) return -1;
+    int sumk = 0;
+    for (int b = 0; b < n_bits; ++b) sumk += 1 << bit_set[b];
+    for (int64_t i = 0; i < rows; ++i) {
+        int wd = row_bits ? (int)row_bits[i] : width, off = 0, found = 0;
+        for (int b = 0; b < n_bits; ++b) {
+            if (bit_set[b] == wd) { found = 1; break; }
+            off += 1 << bit_set[b];
+        }
+        if (!found) return -3;
+        int k = 1 << wd;
+        double c[SKIM_ORACLE_MAX_K];
+        for (int j = 0; j < k; ++j) c[j] = (double)centroids[(size_t)i * sumk + off + j];
+        for (int64_t j = 0; j < cols; ++j) {
+            double x = clustered_value(W[i * ld + j], s, j);
+            int label = nearest_centroid(x, c, k);
+            float cq = centroids[(size_t)i * sumk + off + label];
+            float q = s ? cq * s[j] : cq;
+            float r = half_bits_to_float(W[i * ld + j]) - q;
+            D[i * ldd + j] = float_to_half_bits(ldexpf(r, exp2));
+        }
+    }
+    return 0;
+}
+
+/*
+ * L-full error of every row (Section 3.4, the form the paper names L-full; Section 4.2: "Err refers to the
+ * L-full form"; Algorithm 3, the line that fills the error table):  err_i = d_i H d_i^T  with H = X X^T,
+ * written out as the double sum over j and k in binary64.  D holds the scaled residuals of
+ * skim_oracle_residual (binary16), H [cols][ldh] binary16; the result is divided by 4^exp2.
+ * mag (optional) receives sum_jk |d_j H_jk d_k| / 4^exp2, the scale of the rounding error of any
+ * reduced-precision evaluation.
+ */
+int skim_oracle_err_lfull(const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
+                          int64_t ldh, int exp2, double *err, double *mag)
+{
+    if (!D || !H || !err || rows <= 0 || cols <= 0 || ldd < cols || ldh < cols) return -1;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < rows; ++i) {
+        double *d = (double *)malloc((size_t)cols * sizeof(double));
+        if (!d) { failed = 1; continue; }
+        for (int64_t j = 0; j < cols; ++j) d[j] = (double)half_bits_to_float(D[i * ldd + j]);
+        double acc = 0.0, absacc = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            for (int64_t k = 0; k < cols; ++k) {
+                double t = d[j] * (double)half_bits_to_float(H[j * ldh + k]) * d[k];
+                acc += t;
+                absacc += fabs(t);
+            }
+        }
+        err[i] = ldexp(acc, -2 * exp2);
+        if (mag) mag[i] = ldexp(absacc, -2 * exp2);
+        free(d);
+    }
+    return failed ? -4 : 0;
 }
 
 int skim_oracle_num_threads(void)

@@ -213,6 +213,43 @@ def matvec(em, cols, bit_set, x, s=None):
     return y, mag
 
 
+def residual(W, centroids, bit_set, width=None, row_bits=None, s=None, exp2=8):
+    """Scaled residual float16 [rows, cols]: binary16((float(w) - c[label] * alpha) * 2^exp2); the operand of err_lfull."""
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.float16
+    rows, cols = W.shape
+    centroids = np.ascontiguousarray(centroids, dtype=np.float32)
+    bs, sumk = _bit_array(bit_set)
+    assert centroids.shape == (rows, sumk)
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+    if row_bits is not None:
+        row_bits = np.ascontiguousarray(row_bits, dtype=np.uint8)
+    D = np.zeros((rows, cols), dtype=np.uint16)
+    rc = lib().skim_oracle_residual(_p(W.view(np.uint16)), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols), _p(s),
+                                    _p(row_bits), C.c_int(0 if width is None else int(width)), _p(centroids), _p(bs),
+                                    C.c_int(len(bs)), C.c_int(exp2), _p(D), C.c_int64(cols))
+    if rc:
+        raise ValueError(f"skim_oracle_residual failed ({rc})")
+    return D.view(np.float16)
+
+
+def err_lfull(D, H, exp2=8):
+    """L-full error d H d^T / 4^exp2 of every row of D (float16) for H (float16 [cols, cols]); returns (err, mag)."""
+    D = np.ascontiguousarray(D)
+    H = np.ascontiguousarray(H)
+    assert D.dtype == np.float16 and H.dtype == np.float16
+    rows, cols = D.shape
+    assert H.shape == (cols, cols)
+    err = np.zeros(rows, dtype=np.float64)
+    mag = np.zeros(rows, dtype=np.float64)
+    rc = lib().skim_oracle_err_lfull(_p(D.view(np.uint16)), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols),
+                                     _p(H.view(np.uint16)), C.c_int64(cols), C.c_int(exp2), _p(err), _p(mag))
+    if rc:
+        raise ValueError(f"skim_oracle_err_lfull failed ({rc})")
+    return err, mag
+
+
 def scale_loss_grad(W, importance, labels, alpha, want_grad=True):
     W = np.ascontiguousarray(W)
     assert W.dtype == np.float16

@@ -89,6 +89,21 @@ def make_scale(cols, seed, spread=0.25):
     return np.exp(np.float32(spread) * rng.standard_normal(cols, dtype=np.float32)).astype(np.float32)
 
 
+def make_gram(cols, seed, samples=64, *, correlated=0.3, outlier_channels=4):
+    """A synthetic layer-input Gram matrix H = X X^T / samples (float16 [cols, cols], symmetric) from
+    ``samples`` random input vectors: independent N(0,1) channels plus a shared component of weight
+    ``correlated`` (so off-diagonal entries are not negligible) and a few channels of 8x magnitude, as
+    LLM activations have.  Stands in for calibration activations, which are not available offline."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([int(seed), 0x6A2])))
+    X = rng.standard_normal((cols, samples), dtype=np.float32)
+    X += np.float32(correlated) * rng.standard_normal((1, samples), dtype=np.float32)
+    if outlier_channels:
+        X[rng.choice(cols, size=min(outlier_channels, cols), replace=False)] *= np.float32(8.0)
+    H = (X.astype(np.float64) @ X.astype(np.float64).T) / samples
+    H16 = H.astype(np.float16)
+    return np.ascontiguousarray(np.triu(H16) + np.triu(H16, 1).T)
+
+
 def make_error_table(rows, n_bits, seed, *, monotone=True, ties=False):
     """A synthetic error table (float32 [rows, n_bits]) for allocator tests.
 
