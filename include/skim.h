@@ -20,6 +20,8 @@
  *                         grouping/scaling alternation          (Algorithm 2, outer loop)
  *   skim_scale_update     Adam steps on alpha with the labels fixed
  *                                                               (Algorithm 2, inner repeat)
+ *   skim_residual, skim_err_lfull   the error of a row in the L-full form, (w - wq) X X^T (w - wq)^T
+ *                                                               (Section 3.4; Section 4.2; Algorithm 3)
  *
  * Conventions
  *   - Every array argument is a DEVICE pointer owned by the caller unless its comment says
@@ -267,6 +269,38 @@ int skim_matvec(skim_ctx *ctx, const uint32_t *packed, const int32_t *row_order,
 int skim_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
                       int64_t cols, int64_t ld, const uint8_t *labels, float *alpha, int steps,
                       float lr0, float decay, int decay_every, double *loss_trace);
+
+/*
+ * L-full error (Section 3.4: the layer-wise objective of row i is (w_i - wq_i) X X^T (w_i - wq_i)^T, named
+ * L-full; Section 4.2 and Algorithm 3 use it for the error table; Section 4.3: wq = replace(c, l) * alpha).
+ * Two calls: the residual, then the quadratic form with H = X X^T.
+ *
+ * skim_residual:  D[i][j] = binary16( (float(W_ij) - c_{i,l_ij} * alpha_j) * 2^exp2 )
+ *   label l_ij by the packer's rule (number of midpoints strictly below the clustered value) among the
+ *   centroids of the row's width block; the product c * alpha and the difference are taken in binary32, the
+ *   scaling by 2^exp2 is exact, one rounding to nearest even to binary16 (overflow gives infinity: pick exp2
+ *   so that |residual| * 2^exp2 < 65504; 8 suits weights of magnitude below 1).
+ *   centroids  [rows][sumk] binary32;  row_bits [rows] uint8 or NULL (then every row uses `width`)
+ *   s          the scaling vector alpha itself (device, [cols]) or NULL.  With s != NULL the same vector must be
+ *              installed (skim_apply_scale), else SKIM_ERR_SCALE: the labels need its reciprocal.
+ *   D          out [rows][ldd] binary16, ldd >= cols; for skim_err_lfull: 16-byte aligned, ldd % 8 == 0
+ *   0 <= exp2 <= 24.  A width outside bit_set sets SKIM_STATUS_BAD_BITS and leaves the row untouched.
+ *
+ * skim_err_lfull:  err[i * err_stride] = ( sum_j sum_k D_ij H_jk D_ik ) / 4^exp2
+ *   H          [cols][ldh] binary16 (device), the Gram matrix X X^T of the layer's inputs; only its symmetric
+ *              part matters.  16-byte aligned, ldh % 8 == 0.  cols % 8 == 0.
+ *   scratch    device, 256-byte aligned, at least skim_err_lfull_bytes(rows, cols) bytes
+ *   err        out binary32; err_stride elements between rows (n_bits to fill one column of the error table)
+ * The products are exact in binary32 and are accumulated in binary32 by the tensor cores (cols terms per output
+ * of D H, then cols terms per row), the per-tile sums in binary64:  |err - exact| <= (2 cols + 600) * 2^-24 *
+ * sum_jk |D_ij H_jk D_ik| / 4^exp2.  Needs the workspace (status word).
+ */
+int skim_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *centroids,
+                  const uint8_t *row_bits, int width, const int *bit_set, int n_bits, const float *s, int exp2,
+                  uint16_t *D, int64_t ldd);
+int skim_err_lfull_bytes(int64_t rows, int64_t cols, size_t *out);
+int skim_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
+                   int64_t ldh, int exp2, void *scratch, size_t scratch_bytes, float *err, int64_t err_stride);
 
 /*
  * The whole path from HOST buffers: copies W and importance to the device staging area, runs

@@ -374,6 +374,49 @@ int skim_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance,
                                     loss_trace);
 }
 
+int skim_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *centroids,
+                  const uint8_t *row_bits, int width, const int *bit_set, int n_bits, const float *s, int exp2,
+                  uint16_t *D, int64_t ldd)
+{
+    if (!ctx || !W || !centroids || !D) return SKIM_ERR_NULL;
+    SkimBits bs;
+    int rc = skim_check_bits(bit_set, n_bits, &bs);
+    if (rc) return rc;
+    if (rows < 0 || rows > 0x7fffffff || cols < 1 || cols > 0x7fffff00 || ld < cols || ldd < cols) return SKIM_ERR_SHAPE;
+    if (exp2 < 0 || exp2 > 24) return SKIM_ERR_SHAPE;
+    if (!row_bits && (width < bs.b_min || width > bs.b_max)) return SKIM_ERR_BITSET;
+    rc = check_workspace(ctx, rows, cols);
+    if (rc) return rc;
+    if ((s != nullptr) != ctx->scaled || (ctx->scaled && ctx->scale_cols != cols)) return SKIM_ERR_SCALE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_residual(ctx, W, rows, cols, ld, centroids, row_bits, width, bs, s, exp2, D, ldd);
+}
+
+int skim_err_lfull_bytes(int64_t rows, int64_t cols, size_t *out)
+{
+    if (!out) return SKIM_ERR_NULL;
+    if (rows < 0 || rows > 0x7fffff00 || cols < 8 || cols > 0x7fffff00) return SKIM_ERR_SHAPE;
+    *out = skim_lfull_scratch_bytes(rows, cols);
+    return SKIM_OK;
+}
+
+int skim_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
+                   int64_t ldh, int exp2, void *scratch, size_t scratch_bytes, float *err, int64_t err_stride)
+{
+    if (!ctx || !D || !H || !scratch || !err) return SKIM_ERR_NULL;
+    if (rows < 0 || rows > 0x7fffff00 || cols < 8 || cols > 0x7fffff00 || (cols % 8) != 0) return SKIM_ERR_SHAPE;
+    if (ldd < cols || ldh < cols || (ldd % 8) != 0 || (ldh % 8) != 0 || err_stride < 1) return SKIM_ERR_SHAPE;
+    if (exp2 < 0 || exp2 > 24) return SKIM_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(D) & 15u) || (reinterpret_cast<uintptr_t>(H) & 15u)) return SKIM_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0 || scratch_bytes < skim_lfull_scratch_bytes(rows, cols))
+        return SKIM_ERR_WORKSPACE;
+    if (!ctx->ws) return SKIM_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_err_lfull(ctx, D, rows, cols, ldd, H, ldh, exp2, scratch, err, err_stride);
+}
+
 // ---------------------------------------------------------------- host-buffer path
 
 namespace {

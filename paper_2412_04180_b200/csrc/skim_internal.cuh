@@ -146,6 +146,13 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
                              int64_t cols, int64_t ld, const uint8_t *labels, float *alpha, int steps,
                              float lr0, float decay, int decay_every, double *loss_trace);
 
+int skim_launch_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *centroids,
+                         const uint8_t *row_bits, int width, const SkimBits &bs, const float *s, int exp2, uint16_t *D,
+                         int64_t ldd);
+size_t skim_lfull_scratch_bytes(int64_t rows, int64_t cols);
+int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
+                          int64_t ldh, int exp2, void *scratch, float *err, int64_t err_stride);
+
 __host__ __device__ static inline int64_t skim_row_stride_words(int64_t cols, int b)
 {
     int64_t w = (cols * (int64_t)b + 31) / 32;

@@ -1,0 +1,427 @@
+// L-full error of every row (SKIM Section 3.4: the layer-wise objective written per row,
+// err_i = (w_i - wq_i) X X^T (w_i - wq_i)^T; Section 4.2 and Algorithm 3 fill the error table with it; the
+// paper's scaling vector enters through wq = replace(c, l) * alpha, Section 4.3).
+//
+//   skim_residual_kernel      D = binary16((float(w) - c[label] * alpha) * 2^e): one block per row, labels by the
+//                             same midpoint rule as the packer.  Streaming: 2 B in, 2 B out per element.
+//   skim_lfull_gemm_kernel    Y = D H (H = X X^T, symmetric, binary16) on the tensor cores and, fused into the
+//                             epilogue, the row-wise dot  sum_n Y_in D_in  of every output tile, so Y never
+//                             leaves the SM.  This is the one dense contraction of the method.
+//   skim_lfull_reduce_kernel  adds the per-tile partial sums of a row in a fixed order, divides 4^e out.
+//
+// GEMM kernel: persistent, one CTA per SM, tile 128 x 256 x 64, tcgen05.mma (kind::f16, binary32 accumulators
+// in tensor memory, two accumulator stages of 256 columns), operands brought in by TMA
+// (cp.async.bulk.tensor, 128-byte swizzle) through a 4-stage shared-memory ring.  Warp 0 issues the TMA loads,
+// warp 1 allocates tensor memory and issues the MMAs, warps 2-5 read the accumulators back (tcgen05.ld) and do
+// the dot product with the matching D tile.  No cluster launch and no multicast: every CTA fetches its own tiles.
+// Every wait on an mbarrier is bounded: after WAIT_LIMIT_CYCLES the waiting role raises the block's abort flag,
+// sets SKIM_STATUS_TIMEOUT, and all roles leave their loops; tensor memory is freed on every path.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "skim_internal.cuh"
+
+namespace {
+
+// ---------------------------------------------------------------- residual
+
+constexpr int RES_T = 256;
+
+struct ResidualArgs {
+    const uint16_t *W;
+    const float *rscale;     // 1 / alpha (installed scale), or nullptr
+    const float *s;          // alpha itself, or nullptr
+    const float *centroids;
+    const uint8_t *row_bits; // nullptr: every row at `width`
+    int width;
+    int64_t ld, ldd;
+    int cols;
+    int nb, bmin, sumk;
+    int exp2;
+    uint16_t *D;
+    unsigned long long *status;
+};
+
+__global__ void __launch_bounds__(RES_T) skim_residual_kernel(ResidualArgs a)
+{
+    __shared__ float tf[16];
+    __shared__ float cs[16];
+    const int tid = threadIdx.x;
+    const int64_t row = blockIdx.x;
+    const int b = a.row_bits ? (int)a.row_bits[row] : a.width;
+    const int bi = b - a.bmin;
+    if (bi < 0 || bi >= a.nb) {
+        if (tid == 0) atomicOr(a.status, (unsigned long long)SKIM_STATUS_BAD_BITS);
+        return;
+    }
+    const int k = 1 << b;
+    const int off = (1 << a.bmin) * ((1 << bi) - 1);
+    const float *c = a.centroids + row * a.sumk + off;
+    if (tid < 16) {
+        const float cj = c[min(tid, k - 1)];
+        cs[tid] = cj;
+        float t = __int_as_float(0x7f800000);
+        if (tid < k - 1) {
+            t = __double2float_rd(0.5 * ((double)cj + (double)c[tid + 1]));
+            if (t == 0.0f) t = 0.0f;
+        }
+        tf[tid] = t;
+    }
+    __syncthreads();
+    const uint16_t *Wr = a.W + row * a.ld;
+    uint16_t *Dr = a.D + row * a.ldd;
+    const float scale = __int_as_float((127 + a.exp2) << 23);       // 2^exp2, exact
+    for (int e = tid; e < a.cols; e += RES_T) {
+        const float w = __half2float(__ushort_as_half(Wr[e]));
+        float x = w;
+        if (a.rscale) x = __fmul_rn(w, a.rscale[e]);
+        int code = (x > tf[7]) ? 8 : 0;
+        code += (x > tf[code + 3]) ? 4 : 0;
+        code += (x > tf[code + 1]) ? 2 : 0;
+        code += (x > tf[code]) ? 1 : 0;
+        float q = cs[code];
+        if (a.s) q = __fmul_rn(q, a.s[e]);
+        const float r = __fsub_rn(w, q);
+        Dr[e] = __half_as_ushort(__float2half_rn(__fmul_rn(r, scale)));
+    }
+}
+
+// ---------------------------------------------------------------- GEMM with fused row-wise dot
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;                  // two accumulator stages of BN binary32 columns
+constexpr long long WAIT_LIMIT_CYCLES = 400000000ll;   // about 0.2 s; a whole launch takes milliseconds
+constexpr size_t GEMM_SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+
+struct GemmSync {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok)
+                 : "r"(smem_u32(bar)), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
+// Bounded wait.  False when the block is aborting (this wait ran out, or another role's did).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
+                 : "memory");
+}
+
+// Shared-memory operand descriptor: K-major tile whose rows are 64 binary16 = 128 bytes, 128-byte swizzle,
+// 8-row groups 1024 bytes apart (the layout TMA writes with CU_TENSOR_MAP_SWIZZLE_128B); tiles are 1024-byte
+// aligned, and a step of UMMA_K elements along K inside the swizzle row is a plain 32-byte address offset.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                                // leading byte offset (unused for this layout)
+    d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset: 8 rows x 128 bytes
+    d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                                // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor of kind::f16: D binary32, A and B binary16, both K-major, M = 128, N = 256.
+constexpr uint32_t IDESC = (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+                 "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+                 : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive binary32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *v)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct GemmArgs {
+    const uint16_t *D;       // [rows][ldd] binary16 (also operand A, through its tensor map)
+    int64_t ldd;
+    int rows, cols;
+    int mt, nt;              // tiles along rows and along columns
+    float *partial;          // [mt * BM][nt]
+    unsigned long long *status;
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs a)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *tiles = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    GemmSync &sy = *reinterpret_cast<GemmSync *>(tiles + (size_t)STAGES * STAGE_BYTES);
+    volatile int *abort_flag = &sy.abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = (a.cols + BK - 1) / BK;
+    const int ntiles = a.mt * a.nt;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sy.full[s], 1); mbar_init(&sy.empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sy.tmem_full[s], 1); mbar_init(&sy.tmem_empty[s], 4); }
+        sy.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sy.tmem_base)), "r"(TMEM_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sy.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one lane)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+                const int m0 = (t % a.mt) * BM, n0 = (t / a.mt) * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!(ok = mbar_wait(&sy.empty[stage], phase ^ 1u, abort_flag))) break;
+                    unsigned char *sa = tiles + (size_t)stage * STAGE_BYTES;
+                    mbar_expect_tx(&sy.full[stage], STAGE_BYTES);
+                    tma_load_2d(sa, &map_a, &sy.full[stage], kb * BK, m0);
+                    tma_load_2d(sa + A_BYTES, &map_b, &sy.full[stage], kb * BK, n0);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
+                const int as = it & 1;
+                if (!(ok = mbar_wait(&sy.tmem_empty[as], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!(ok = mbar_wait(&sy.full[stage], phase, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(tiles + (size_t)stage * STAGE_BYTES), sb = sa + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_f16(tmem_d, umma_desc(sa + k * UMMA_K * 2), umma_desc(sb + k * UMMA_K * 2), (kb | k) ? 1u : 0u);
+                    umma_commit(&sy.empty[stage]);           // the stage is free once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(&sy.tmem_full[as]);      // the accumulator is complete once all MMAs are
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: 4 warps, one row per thread
+        const int q = warp & 3;                               // the tensor-memory lane quarter this warp may read
+        bool ok = true;
+        int it = 0;
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
+            const int as = it & 1;
+            const int mb = t % a.mt, nb = t / a.mt;
+            const int row = mb * BM + q * 32 + lane;
+            const int n0 = nb * BN;
+            const uint16_t *drow = a.D + (int64_t)min(row, a.rows - 1) * a.ldd;
+            ok = mbar_wait(&sy.tmem_full[as], ((uint32_t)it >> 1) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float acc = 0.0f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col = n0 + c * 32;
+                uint4 dv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    dv[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (col + u * 8 + 8 <= a.cols) dv[u] = __ldg(reinterpret_cast<const uint4 *>(drow + col + u * 8));
+                }
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32), v);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t w4[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w4[h]));
+                        acc = fmaf(__uint_as_float(v[u * 8 + 2 * h]), f.x, acc);
+                        acc = fmaf(__uint_as_float(v[u * 8 + 2 * h + 1]), f.y, acc);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sy.tmem_empty[as]);
+            if (row < a.rows) a.partial[(int64_t)row * a.nt + nb] = acc;
+        }
+    }
+    // ---------------------------------------------------------------- teardown (every path comes here)
+    tc_fence_before();
+    __syncthreads();
+    if (sy.abort) {
+        // a wait ran out: give the bulk copies that may still be in flight time to land before the block's
+        // shared memory is released (about a millisecond), and report
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0) atomicOr(a.status, (unsigned long long)SKIM_STATUS_TIMEOUT);
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS));
+    }
+}
+
+__global__ void skim_lfull_reduce_kernel(const float *__restrict__ partial, int rows, int nt, int exp2, float *__restrict__ err,
+                                         int64_t err_stride)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows) return;
+    double s = 0.0;
+    for (int t = 0; t < nt; ++t) s += (double)partial[(int64_t)i * nt + t];
+    err[(int64_t)i * err_stride] = (float)ldexp(s, -2 * exp2);
+}
+
+int encode_map(CUtensorMap *map, const uint16_t *base, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+{
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn)
+        return SKIM_ERR_CUDA;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn)(
+        map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<uint16_t *>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SKIM_OK : SKIM_ERR_CUDA;
+}
+
+}  // namespace
+
+int skim_launch_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *centroids,
+                         const uint8_t *row_bits, int width, const SkimBits &bs, const float *s, int exp2, uint16_t *D,
+                         int64_t ldd)
+{
+    if (rows == 0) return SKIM_OK;
+    SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
+    ResidualArgs a;
+    a.W = W;
+    a.rscale = ctx->scaled ? ws.rscale : nullptr;
+    a.s = s;
+    a.centroids = centroids;
+    a.row_bits = row_bits;
+    a.width = width;
+    a.ld = ld;
+    a.ldd = ldd;
+    a.cols = (int)cols;
+    a.nb = bs.n_bits;
+    a.bmin = bs.b_min;
+    a.sumk = bs.sumk;
+    a.exp2 = exp2;
+    a.D = D;
+    a.status = ws.status;
+    skim_residual_kernel<<<(unsigned)rows, RES_T, 0, ctx->stream>>>(a);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    return SKIM_OK;
+}
+
+size_t skim_lfull_scratch_bytes(int64_t rows, int64_t cols)
+{
+    const int64_t mt = (rows + BM - 1) / BM, nt = (cols + BN - 1) / BN;
+    return skim_align256((size_t)(mt * BM) * (size_t)nt * sizeof(float));
+}
+
+int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
+                          int64_t ldh, int exp2, void *scratch, float *err, int64_t err_stride)
+{
+    if (rows == 0) return SKIM_OK;
+    CUtensorMap map_a, map_b;
+    int rc = encode_map(&map_a, D, rows, cols, ldd, BM);
+    if (rc) return rc;
+    rc = encode_map(&map_b, H, cols, cols, ldh, BN);
+    if (rc) return rc;
+    GemmArgs a;
+    a.D = D;
+    a.ldd = ldd;
+    a.rows = (int)rows;
+    a.cols = (int)cols;
+    a.mt = (int)((rows + BM - 1) / BM);
+    a.nt = (int)((cols + BN - 1) / BN);
+    a.partial = (float *)scratch;
+    a.status = (unsigned long long *)ctx->ws;
+    SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lfull_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
+    const int tiles = a.mt * a.nt;
+    const unsigned blocks = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);    // persistent: one CTA per SM
+    skim_lfull_gemm_kernel<<<blocks, GEMM_THREADS, GEMM_SMEM, ctx->stream>>>(map_a, map_b, a);
+    SKIM_CUDA_OK(cudaGetLastError());
+    skim_lfull_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, ctx->stream>>>(a.partial, (int)rows, a.nt, exp2, err, err_stride);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 2;
+    return SKIM_OK;
+}

@@ -22,7 +22,7 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
            "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_bits_until", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
-           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_host_staging_bytes",
+           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_residual", "skim_err_lfull_bytes", "skim_err_lfull", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
            "skim_kernel_times", "skim_early_exit", "skim_lloyd_iterations", "skim_strerror"]
 
@@ -281,6 +281,44 @@ class Skim:
                                      C.c_int64(cols), _ptr(labels), _ptr(alpha), C.c_int(steps), C.c_float(lr0),
                                      C.c_float(decay), C.c_int(decay_every), _ptr(trace)), "skim_scale_update")
         return trace[:steps] if want_trace else None
+
+    def residual(self, W, centroids, bit_set, width=None, row_bits=None, s=None, exp2=8, out=None):
+        """float16 [rows, cols] scaled residual (W - c[label] * alpha) * 2^exp2, the operand of err_lfull."""
+        _dev(W, torch.float16, "W")
+        _dev(centroids, torch.float32, "centroids")
+        rows, cols = W.shape
+        arr, nb, _ = _bits(bit_set)
+        if row_bits is not None:
+            _dev(row_bits, torch.uint8, "row_bits")
+        if s is not None:
+            _dev(s, torch.float32, "s")
+        if out is None:
+            out = torch.empty((rows, cols), dtype=torch.float16, device=W.device)
+        _chk(lib().skim_residual(self._h, _ptr(W), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols), _ptr(centroids),
+                                 _ptr(row_bits), C.c_int(0 if width is None else int(width)), arr, C.c_int(nb), _ptr(s),
+                                 C.c_int(exp2), _ptr(out), C.c_int64(out.stride(0))), "skim_residual")
+        return out
+
+    @staticmethod
+    def err_lfull_bytes(rows, cols):
+        out = C.c_size_t()
+        _chk(lib().skim_err_lfull_bytes(C.c_int64(rows), C.c_int64(cols), C.byref(out)), "skim_err_lfull_bytes")
+        return out.value
+
+    def err_lfull(self, D, H, exp2=8, scratch=None, out=None, out_stride=1):
+        """float32 [rows] L-full errors d H d^T / 4^exp2 of the rows of D (float16) for H (float16 [cols, cols])."""
+        _dev(D, torch.float16, "D")
+        _dev(H, torch.float16, "H")
+        rows, cols = D.shape
+        need = self.err_lfull_bytes(rows, cols)
+        if scratch is None:
+            scratch = torch.empty(need, dtype=torch.uint8, device=D.device)
+        if out is None:
+            out = torch.empty((rows,), dtype=torch.float32, device=D.device)
+        _chk(lib().skim_err_lfull(self._h, _ptr(D), C.c_int64(rows), C.c_int64(cols), C.c_int64(D.stride(0)), _ptr(H),
+                                  C.c_int64(H.stride(0)), C.c_int(exp2), _ptr(scratch), C.c_size_t(scratch.numel()),
+                                  _ptr(out), C.c_int64(out_stride)), "skim_err_lfull")
+        return out
 
     @staticmethod
     def host_staging_bytes(rows, cols, bit_set):
