@@ -681,6 +681,118 @@ int skim_oracle_scale_update(const uint16_t *W, const float *importance, int64_t
     return rc;
 }
 
+/* ------------------------------------------------------------------ exact 1-D weighted K-means */
+
+typedef struct { double x, g; } oracle_pair;
+
+static int cmp_pair(const void *a, const void *b)
+{
+    double x = ((const oracle_pair *)a)->x, y = ((const oracle_pair *)b)->x;
+    return (x > y) - (x < y);
+}
+
+/*
+ * The optimum of the clustering objective of Section 3.2 (diagonal form), sum_j g_j (x_j - c_{l_j})^2, over ALL
+ * assignments to k centroids, for one row: in one dimension the optimal clusters are intervals of the sorted
+ * row, so the textbook dynamic programme over split points finds it,
+ *     F_1(i) = cost(0, i),   F_j(i) = min_{j-1 <= t < i} F_{j-1}(t) + cost(t, i),
+ *     cost(t, i) = sum g x^2 - (sum g x)^2 / sum g  over the sorted elements t .. i-1 (0 without weight),
+ * every t tried (no monotonicity assumed), smallest t on ties.  This is the yardstick for the Lloyd
+ * iterations of Algorithm 3, which only reach a local optimum.
+ *   ks [nk] ascending cluster counts; c out: concatenated blocks of ks[u] centroids (weighted means of the
+ *   intervals, ascending; an interval without weight takes the mean of its first and last value);
+ *   err out [nk]: the optimum.  A row with D <= k distinct values gets them as centroids, padded with the
+ *   largest, and err = 0, as in skim_oracle_kmeans_row.
+ */
+int skim_oracle_kmeans_exact_row(const double *x, const double *g, int64_t m, const int *ks, int nk, double *c, double *err)
+{
+    if (!x || !g || !ks || !c || !err || m <= 0 || nk <= 0) return -1;
+    int kmax = ks[nk - 1];
+    if (kmax > SKIM_ORACLE_MAX_K) return -1;
+    oracle_pair *v = (oracle_pair *)malloc((size_t)m * sizeof(oracle_pair));
+    double *p0 = (double *)malloc((size_t)(m + 1) * 3 * sizeof(double));
+    if (!v || !p0) { free(v); free(p0); return -1; }
+    double *p1 = p0 + (m + 1), *p2 = p1 + (m + 1);
+    for (int64_t j = 0; j < m; ++j) { v[j].x = (x[j] == 0.0) ? 0.0 : x[j]; v[j].g = g[j]; }
+    qsort(v, (size_t)m, sizeof(oracle_pair), cmp_pair);
+    p0[0] = p1[0] = p2[0] = 0.0;
+    int64_t distinct = 1;
+    for (int64_t j = 0; j < m; ++j) {
+        p0[j + 1] = p0[j] + v[j].g;
+        p1[j + 1] = p1[j] + v[j].g * v[j].x;
+        p2[j + 1] = p2[j] + v[j].g * v[j].x * v[j].x;
+        if (j && v[j].x != v[j - 1].x) ++distinct;
+    }
+    int64_t limit = (int64_t)kmax < m ? (int64_t)kmax : m;      /* layers that can have non-empty intervals */
+    double *F = (double *)malloc((size_t)(limit + 1) * (size_t)(m + 1) * sizeof(double));
+    int32_t *T = (int32_t *)malloc((size_t)(limit + 1) * (size_t)(m + 1) * sizeof(int32_t));
+    if (!F || !T) { free(v); free(p0); free(F); free(T); return -1; }
+#define COST(t, i) ((p0[i] - p0[t]) > 0.0 ? (p2[i] - p2[t]) - (p1[i] - p1[t]) * (p1[i] - p1[t]) / (p0[i] - p0[t]) : 0.0)
+    for (int64_t i = 1; i <= m; ++i) { F[1 * (m + 1) + i] = COST(0, i); T[1 * (m + 1) + i] = 0; }
+    for (int64_t j = 2; j <= limit; ++j) {
+        for (int64_t i = j; i <= m; ++i) {
+            double best = 0.0;
+            int64_t bt = -1;
+            for (int64_t t = j - 1; t < i; ++t) {
+                double val = F[(j - 1) * (m + 1) + t] + COST(t, i);
+                if (bt < 0 || val < best) { best = val; bt = t; }
+            }
+            F[j * (m + 1) + i] = best;
+            T[j * (m + 1) + i] = (int32_t)bt;
+        }
+    }
+#undef COST
+    int off = 0;
+    for (int u = 0; u < nk; ++u) {
+        int k = ks[u];
+        if (distinct <= (int64_t)k) {
+            int q = 0;
+            for (int64_t j = 0; j < m; ++j)
+                if (j == 0 || v[j].x != v[j - 1].x) c[off + q++] = v[j].x;
+            for (; q < k; ++q) c[off + q] = v[m - 1].x;
+            err[u] = 0.0;
+        } else {
+            int64_t i = m;
+            for (int j = k; j >= 1; --j) {
+                int64_t t = (j == 1) ? 0 : T[(int64_t)j * (m + 1) + i];
+                double s0 = p0[i] - p0[t];
+                c[off + j - 1] = s0 > 0.0 ? (p1[i] - p1[t]) / s0 : 0.5 * (v[t].x + v[i - 1].x);
+                i = t;
+            }
+            double e = F[(int64_t)k * (m + 1) + m];
+            err[u] = e > 0.0 ? e : 0.0;
+        }
+        off += k;
+    }
+    free(v); free(p0); free(F); free(T);
+    return 0;
+}
+
+/* Exact clustering of every row of a matrix at every width of bit_set (the counterpart of
+ * skim_oracle_cluster_rows with the Lloyd iterations replaced by the optimum). */
+int skim_oracle_cluster_rows_exact(const uint16_t *W, const float *importance, int64_t rows, int64_t cols, int64_t ld,
+                                   const float *s, const int *bit_set, int n_bits, double *centroids, double *err)
+{
+    if (!W || !importance || !centroids || !err || rows <= 0 || cols <= 0 || ld < cols) return -1;
+    if (check_bit_set(bit_set, n_bits)) return -1;
+    int ks[8], sumk = 0;
+    for (int b = 0; b < n_bits; ++b) { ks[b] = 1 << bit_set[b]; sumk += ks[b]; }
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < rows; ++i) {
+        double *x = (double *)malloc((size_t)cols * 2 * sizeof(double));
+        if (!x) { failed = 1; continue; }
+        double *g = x + cols;
+        for (int64_t j = 0; j < cols; ++j) {
+            x[j] = clustered_value(W[i * ld + j], s, j);
+            g[j] = (double)importance[i * ld + j];
+        }
+        if (skim_oracle_kmeans_exact_row(x, g, cols, ks, n_bits, centroids + (size_t)i * sumk, err + (size_t)i * n_bits)) failed = 1;
+        free(x);
+    }
+    return failed ? -4 : 0;
+}
+
 /* ------------------------------------------------------------------ L-full error (Section 3.4) */
 
 /*

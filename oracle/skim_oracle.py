@@ -103,6 +103,38 @@ def cluster_rows(W, importance, bit_set, iters, s=None, row_bits=None, round_fp3
     return dict(centroids=centroids, codes=codes, err=err, trace=trace)
 
 
+def kmeans_exact_row(x, g, ks):
+    """Optimal weighted 1-D K-means of one row for every cluster count in ``ks`` (ascending): returns
+    (centroids: concatenated blocks, err [len(ks)])."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    ks = np.ascontiguousarray(ks, dtype=np.int32)
+    c = np.zeros(int(ks.sum()), dtype=np.float64)
+    err = np.zeros(len(ks), dtype=np.float64)
+    rc = lib().skim_oracle_kmeans_exact_row(_p(x), _p(g), C.c_int64(x.shape[0]), _p(ks), C.c_int(len(ks)), _p(c), _p(err))
+    if rc:
+        raise ValueError(f"skim_oracle_kmeans_exact_row failed ({rc})")
+    return c, err
+
+
+def cluster_rows_exact(W, importance, bit_set, s=None):
+    """Exact (optimal) clustering of all rows at all widths: dict(centroids float64 [rows, sum 2^b], err [rows, n_bits])."""
+    W = np.ascontiguousarray(W)
+    assert W.dtype == np.float16 and W.ndim == 2
+    importance = np.ascontiguousarray(importance, dtype=np.float32)
+    rows, cols = W.shape
+    bits, sumk = _bit_array(bit_set)
+    if s is not None:
+        s = np.ascontiguousarray(s, dtype=np.float32)
+    centroids = np.zeros((rows, sumk), dtype=np.float64)
+    err = np.zeros((rows, len(bits)), dtype=np.float64)
+    rc = lib().skim_oracle_cluster_rows_exact(_p(W.view(np.uint16)), _p(importance), C.c_int64(rows), C.c_int64(cols),
+                                              C.c_int64(cols), _p(s), _p(bits), C.c_int(len(bits)), _p(centroids), _p(err))
+    if rc:
+        raise ValueError(f"skim_oracle_cluster_rows_exact failed ({rc})")
+    return dict(centroids=centroids, err=err)
+
+
 def allocate_bits(err, b_min, budget, floor_start=False, round_up=False):
     """Greedy allocation over a float32 table [rows, n_bits]; returns (bits uint8 [rows], total).
     floor_start: every row starts at floor(budget) instead of b_min.  round_up: Algorithm 1's literal
