@@ -20,6 +20,7 @@
  *                         grouping/scaling alternation          (Algorithm 2, outer loop)
  *   skim_scale_update     Adam steps on alpha with the labels fixed
  *                                                               (Algorithm 2, inner repeat)
+ *   skim_cluster_rows_exact  the optimum of the clustering objective per row (yardstick for the iterations)
  *   skim_residual, skim_err_lfull   the error of a row in the L-full form, (w - wq) X X^T (w - wq)^T
  *                                                               (Section 3.4; Section 4.2; Algorithm 3)
  *
@@ -124,6 +125,25 @@ int skim_cluster_rows(skim_ctx *ctx, const uint16_t *W, const float *importance,
 int skim_cluster_rows_at(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
                          int64_t cols, int64_t ld, const uint8_t *row_bits, const int *bit_set,
                          int n_bits, int iters, float *centroids, uint8_t *codes, float *err);
+
+/*
+ * The optimum of the clustering objective (Section 3.2, diagonal form: sum_j g_ij (x_ij - c)^2 over all
+ * assignments to 2^b centroids), where skim_cluster_rows runs the Lloyd iterations of Algorithm 3, which stop
+ * in a local optimum: the yardstick for them, at the same interface.  In one dimension the optimal clusters are
+ * intervals of the sorted row; a dynamic programme over the split points finds them (cols * log cols cost
+ * evaluations per centroid, all widths sharing the layers).
+ *   centroids  out [rows][sumk] binary32: the weighted means of the optimal intervals, ascending (an interval
+ *              whose importances are all zero takes the mean of its first and last value)
+ *   err        out [rows][n_bits] binary32: the optimum
+ * Rows with at most 2^b distinct values get those values and error 0, as in skim_cluster_rows.  Where two
+ * partitions cost the same up to rounding either may be returned.  An installed scale vector applies.
+ *   scratch    device, 256-byte aligned, at least skim_cluster_exact_bytes(ctx, rows, cols) bytes
+ *              (about 74 bytes per column for each of min(rows, 3 x SM count) rows in flight)
+ */
+int skim_cluster_exact_bytes(const skim_ctx *ctx, int64_t rows, int64_t cols, size_t *out);
+int skim_cluster_rows_exact(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                            int64_t ld, const int *bit_set, int n_bits, void *scratch, size_t scratch_bytes,
+                            float *centroids, float *err);
 
 /*
  * Algorithm 1.  All rows start at b_min; the row with the largest error reduction

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libskim.so")
 LIB_CHECKED = os.path.join(HERE, "libskim_checked.so")   # the same sources with -DSKIM_CHECK_BOUNDS
-SOURCES = ["skim_api.cu", "skim_cluster.cu", "skim_cluster16.cu", "skim_lloyd.cu", "skim_allocate.cu", "skim_quantize.cu", "skim_unpack.cu", "skim_scale.cu", "skim_lfull.cu"]
+SOURCES = ["skim_api.cu", "skim_cluster.cu", "skim_cluster16.cu", "skim_lloyd.cu", "skim_allocate.cu", "skim_quantize.cu", "skim_unpack.cu", "skim_scale.cu", "skim_lfull.cu", "skim_exact.cu"]
 
 
 def _stale(lib=LIB) -> bool:

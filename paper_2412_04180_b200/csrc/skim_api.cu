@@ -187,6 +187,36 @@ int skim_cluster_rows_at(skim_ctx *ctx, const uint16_t *W, const float *importan
     return cluster_common(ctx, W, importance, rows, cols, ld, row_bits, bit_set, n_bits, iters, centroids, codes, err);
 }
 
+int skim_cluster_exact_bytes(const skim_ctx *ctx, int64_t rows, int64_t cols, size_t *out)
+{
+    if (!ctx || !out) return SKIM_ERR_NULL;
+    int rc = check_matrix(ctx, rows, cols, cols);
+    if (rc) return rc;
+    *out = skim_align256((size_t)skim_exact_slots(ctx, rows > 0 ? rows : 1) * skim_exact_slot_bytes(cols));
+    return SKIM_OK;
+}
+
+int skim_cluster_rows_exact(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                            int64_t ld, const int *bit_set, int n_bits, void *scratch, size_t scratch_bytes,
+                            float *centroids, float *err)
+{
+    if (!ctx || !W || !importance || !scratch || !centroids || !err) return SKIM_ERR_NULL;
+    SkimBits bits;
+    int rc = skim_check_bits(bit_set, n_bits, &bits);
+    if (rc) return rc;
+    rc = check_matrix(ctx, rows, cols, ld);
+    if (rc) return rc;
+    rc = check_workspace(ctx, rows, cols);
+    if (rc) return rc;
+    if (ctx->scaled && ctx->scale_cols != cols) return SKIM_ERR_SCALE;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0 ||
+        scratch_bytes < (size_t)skim_exact_slots(ctx, rows > 0 ? rows : 1) * skim_exact_slot_bytes(cols))
+        return SKIM_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_cluster(ctx, W, importance, rows, cols, ld, nullptr, bits, 0, centroids, nullptr, err, scratch);
+}
+
 int skim_allocate_bits(skim_ctx *ctx, const float *err, int64_t rows, const int *bit_set, int n_bits, double budget,
                        uint8_t *bits_out, int64_t *total_bits)
 {

@@ -234,7 +234,7 @@ int skim_cluster_max_cols(int max_smem_optin, int64_t *out)
 
 int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
                         int64_t cols, int64_t ld, const uint8_t *row_bits, const SkimBits &bits,
-                        int iters, float *centroids, uint8_t *codes, float *err)
+                        int iters, float *centroids, uint8_t *codes, float *err, void *exact_scratch)
 {
     if (rows == 0) return SKIM_OK;
     SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
@@ -287,7 +287,8 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
             ctx->launches += 1;
         }
         if (tev) SKIM_CUDA_OK(cudaEventRecord(tev[1], ctx->stream));
-        const int rc = skim_launch_lloyd(ctx, a, n);
+        const int rc = exact_scratch ? skim_launch_exact(ctx, a, n, exact_scratch, skim_exact_slots(ctx, rows))
+                                     : skim_launch_lloyd(ctx, a, n);
         if (rc) return rc;
         if (tev) {
             SKIM_CUDA_OK(cudaEventRecord(tev[2], ctx->stream));

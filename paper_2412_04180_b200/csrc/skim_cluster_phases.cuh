@@ -343,5 +343,8 @@ __device__ __forceinline__ void write_distinct_values(const ClusterArgs &a, int 
 // is false (planning) and launches over `rows` rows otherwise.  Returns SKIM_OK, or 1 when the
 // call does not meet the kernel's requirements (then the generic sort kernel must be used).
 int skim_launch_sort16(skim_ctx *ctx, skimk::ClusterArgs &args, int64_t rows, bool launch);
+// Exact clustering kernel (skim_exact.cu): one block per row record; `scratch` holds `slots` slots of
+// skim_exact_slot_bytes(cols) bytes.
+int skim_launch_exact(skim_ctx *ctx, const skimk::ClusterArgs &args, int64_t rows, void *scratch, int slots);
 // Lloyd kernel (skim_lloyd.cu): one warp per row record.
 int skim_launch_lloyd(skim_ctx *ctx, const skimk::ClusterArgs &args, int64_t rows);

@@ -123,9 +123,12 @@ int skim_check_bits(const int *bit_set, int n_bits, SkimBits *out);
     } while (0)
 
 // Launchers implemented in the kernel translation units.  All return SKIM_OK or SKIM_ERR_*.
+// exact_scratch == nullptr: Lloyd iterations (Algorithm 3); else the exact optimum of every row (skim_exact.cu)
 int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows,
                         int64_t cols, int64_t ld, const uint8_t *row_bits, const SkimBits &bits,
-                        int iters, float *centroids, uint8_t *codes, float *err);
+                        int iters, float *centroids, uint8_t *codes, float *err, void *exact_scratch = nullptr);
+size_t skim_exact_slot_bytes(int64_t cols);
+int skim_exact_slots(const skim_ctx *ctx, int64_t rows);
 int skim_cluster_max_cols(int max_smem_optin, int64_t *out);
 int skim_launch_reciprocal(skim_ctx *ctx, const float *s, int64_t cols);
 int skim_launch_allocate(skim_ctx *ctx, const float *err, int64_t rows, const SkimBits &bits, int first_col,

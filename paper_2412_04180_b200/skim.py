@@ -21,7 +21,7 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
              -7: "SKIM_ERR_BAD_DATA", -8: "SKIM_ERR_SCALE", -9: "SKIM_ERR_ALIGN", -10: "SKIM_ERR_STATIC_LIMIT"}
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
-           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_bits_until", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
+           "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_cluster_exact_bytes", "skim_cluster_rows_exact", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_bits_until", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
            "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_residual", "skim_err_lfull_bytes", "skim_err_lfull", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
            "skim_kernel_times", "skim_early_exit", "skim_lloyd_iterations", "skim_strerror"]
@@ -178,6 +178,23 @@ class Skim:
                                         C.c_int64(cols), _ptr(row_bits), arr, C.c_int(nb), C.c_int(iters),
                                         _ptr(cent), _ptr(codes), _ptr(err)), "skim_cluster_rows_at")
         return cent, codes, err
+
+    def cluster_rows_exact(self, W, importance, bit_set, scratch=None):
+        """The optimum of the clustering objective per row: returns (centroids [rows, sumk], err [rows, n_bits])."""
+        _dev(W, torch.float16, "W")
+        _dev(importance, torch.float32, "importance")
+        rows, cols = W.shape
+        arr, nb, sumk = _bits(bit_set)
+        need = C.c_size_t()
+        _chk(lib().skim_cluster_exact_bytes(self._h, C.c_int64(rows), C.c_int64(cols), C.byref(need)), "skim_cluster_exact_bytes")
+        if scratch is None:
+            scratch = torch.empty(need.value, dtype=torch.uint8, device=W.device)
+        cent = torch.empty((rows, sumk), dtype=torch.float32, device=W.device)
+        err = torch.empty((rows, nb), dtype=torch.float32, device=W.device)
+        _chk(lib().skim_cluster_rows_exact(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
+                                           C.c_int64(cols), arr, C.c_int(nb), _ptr(scratch), C.c_size_t(scratch.numel()),
+                                           _ptr(cent), _ptr(err)), "skim_cluster_rows_exact")
+        return cent, err
 
     def allocate_bits(self, err, bit_set, budget, out=None, floor_start=False, round_up=False):
         """Returns (bits uint8 [rows], total_bits).  floor_start: every row starts at floor(budget)
