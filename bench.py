@@ -54,6 +54,16 @@ def measured_peak():
         return 6650.0, "fallback"
 
 
+def measured_tensor_peak():
+    """Measured dense bf16 tensor throughput (TFLOP/s) for a kernel timed alone; fp16 runs at the same rate."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (cuBLAS bf16 burst; fp16 has the same nominal rate)"
+    except Exception:
+        return 1590.0, "fallback"
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -359,6 +369,54 @@ def run_ours(args):
         # the pipeline's own outputs again (the round above overwrote the packed form with the scaled one)
         step()
         stream.synchronize()
+
+        # the error table in the paper's L-full form on the same matrix (outside the timed region): residual +
+        # tcgen05 GEMM with the row-wise dot fused in, once per width, against a synthetic Gram matrix
+        tpeak, tpeak_kind = measured_tensor_peak()
+        with torch.cuda.stream(stream):
+            Hc = torch.from_numpy(inputs.make_gram(COLS, SEED + 7)).cuda()
+            Dbuf = torch.empty((ROWS, COLS), dtype=torch.float16, device="cuda")
+            lf_scr = torch.empty(ctx.err_lfull_bytes(ROWS, COLS), dtype=torch.uint8, device="cuda")
+            table = torch.empty((ROWS, nb), dtype=torch.float32, device="cuda")
+            for _ in range(2):
+                ctx.residual(W, cent, BIT_SET, width=BIT_SET[-1], out=Dbuf)
+                ctx.err_lfull(Dbuf, Hc, scratch=lf_scr, out=table[:, nb - 1], out_stride=nb)
+            l0, l1, l2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            res_ms = gemm_ms = 0.0
+            for bi, b in enumerate(BIT_SET):
+                l0.record(stream)
+                ctx.residual(W, cent, BIT_SET, width=b, out=Dbuf)
+                l1.record(stream)
+                ctx.err_lfull(Dbuf, Hc, scratch=lf_scr, out=table[:, bi], out_stride=nb)
+                l2.record(stream)
+                stream.synchronize()
+                res_ms += l0.elapsed_time(l1)
+                gemm_ms += l1.elapsed_time(l2)
+            assert ctx.get_status() == 0 and bool(torch.isfinite(table).all())
+        flops = 2.0 * ROWS * COLS * COLS
+        extra["lfull_table"] = {"residual_ms_per_width": res_ms / nb, "gemm_ms_per_width": gemm_ms / nb,
+                                "table_ms_all_widths": res_ms + gemm_ms,
+                                "roofline": {"bound": "tensor", "kernel": "skim_lfull_gemm_kernel", "dtype": "fp16 in, fp32 accumulate",
+                                             "achieved": flops / (gemm_ms / nb * 1e-3) / 1e12, "peak": tpeak, "peak_kind": f"of {tpeak_kind}",
+                                             "unit": "TFLOP/s", "frac": flops / (gemm_ms / nb * 1e-3) / 1e12 / tpeak, "traffic": None},
+                                "note": "Section 3.4's L-full error for every row and width: 2*rows*cols^2 flop per width"}
+        del Hc, Dbuf, lf_scr
+
+        # the optimum of the clustering objective per row (yardstick for the 50 Lloyd iterations)
+        with torch.cuda.stream(stream):
+            need = torch.empty(0)
+            x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ctx.cluster_rows_exact(W[:296], G[:296], BIT_SET)
+            x0.record(stream)
+            _, err_opt = ctx.cluster_rows_exact(W, G, BIT_SET)
+            x1.record(stream)
+            stream.synchronize()
+            ratio = (err_opt.double() / err.double().clamp_min(1e-300)).cpu().numpy()
+        extra["exact_clustering"] = {"ms": x0.elapsed_time(x1),
+                                     "optimum_over_lloyd_error_mean_per_width": [float(v) for v in ratio.mean(axis=0)],
+                                     "optimum_over_lloyd_error_median_per_width": [float(v) for v in np.median(ratio, axis=0)],
+                                     "note": "skim_cluster_rows_exact on the same matrix: the iterations' error table entries "
+                                             "divided into the optimum's (1.0 = the iterations found the optimum)"}
 
     # the consumers of the packed form (outside the timed region; reported beside the step)
     consumers = None

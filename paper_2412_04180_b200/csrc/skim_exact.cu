@@ -11,9 +11,10 @@
 //   prefix   the record's two-level prefix sums become one flat array Q[t] = (P0, P1, P2, F_{j-1})(t): a cost
 //            evaluation is one 32-byte load.
 //   layer    positions are visited like the in-order nodes of a perfect binary tree, level by level: a node's
-//            search range is bounded by the minimisers of its two nearest finished neighbours.  The first
-//            levels have few nodes with long ranges (a group of threads shares a node and reduces), the last
-//            ones many nodes with short ranges (one thread per node).
+//            search range is bounded by the minimisers of its two nearest finished neighbours.  The ranges of
+//            a level tile the span of split points; the span is dealt to the threads in equal stretches and
+//            the candidates of a node meet in one atomic minimum, because the ranges themselves are very
+//            unequal (the minimiser jumps where an outlier enters the prefix).
 //   result   for every width the split points are walked back from the row's end; centroid = weighted mean of
 //            its interval (an interval without weight: mean of its first and last value), error = F_k(m).
 // All widths share the layers: F_2, F_4, F_8, F_16 are read off on the way.
@@ -43,11 +44,31 @@ __host__ __device__ inline ExactSlot exact_slot(int m)
     return S;
 }
 
+// shared memory: the minimisers by tree position (2^L + 8 entries, 2^L - 1 >= m), then one key per node of a level
+__host__ __device__ inline size_t exact_optarr_bytes(int m)
+{
+    int L = 1;
+    while ((1 << L) - 1 < m) ++L;
+    return ((((size_t)1 << L) + 8) * sizeof(uint16_t) + 15) & ~(size_t)15;
+}
+__host__ __device__ inline size_t exact_smem_bytes(int m) { return exact_optarr_bytes(m) + ((size_t)m / 2 + 8) * sizeof(unsigned long long); }
+
 __device__ __forceinline__ double4 ld_q(const double4 *p)
 {
     double4 v;
     asm volatile("ld.global.v4.f64 {%0, %1, %2, %3}, [%4];" : "=d"(v.x), "=d"(v.y), "=d"(v.z), "=d"(v.w) : "l"(p));
     return v;
+}
+
+// Candidates of one node compete through a 64-bit atomic minimum: the order-preserving image of the cost with
+// its 16 lowest mantissa bits replaced by the split point, so that costs equal to 2^-36 relative go to the
+// smaller split point.
+__device__ __forceinline__ unsigned long long candidate_key(double v, int t)
+{
+    if (v == 0.0) v = 0.0;
+    const unsigned long long u = (unsigned long long)__double_as_longlong(v);
+    const unsigned long long ob = (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+    return (ob & ~0xffffull) | (unsigned long long)(unsigned)t;
 }
 
 // cost of the interval [t, i) given Q[t] and Q[i]
@@ -60,8 +81,6 @@ __device__ __forceinline__ double interval_cost(const double4 &qt, const double4
 __global__ void __launch_bounds__(XT) skim_exact_kernel(ClusterArgs a, int rows_in_chunk, unsigned char *scratch, size_t slot_bytes)
 {
     extern __shared__ __align__(16) unsigned char xsmem[];
-    __shared__ double sval[XT];
-    __shared__ int sarg[XT];
     __shared__ float s_dvals[16];
     const int tid = threadIdx.x;
     const int m = a.m;
@@ -72,6 +91,7 @@ __global__ void __launch_bounds__(XT) skim_exact_kernel(ClusterArgs a, int rows_
     double *Fc = reinterpret_cast<double *>(slot + S.fc);
     uint16_t *T = reinterpret_cast<uint16_t *>(slot + S.t);
     uint16_t *optarr = reinterpret_cast<uint16_t *>(xsmem);           // minimisers of the current layer by node position
+    unsigned long long *keys = reinterpret_cast<unsigned long long *>(xsmem + exact_optarr_bytes(m));   // per node of a level
     const int kmax = 1 << (a.bmin + a.nb - 1);
 
     for (int local = blockIdx.x; local < rows_in_chunk; local += gridDim.x) {
@@ -125,70 +145,84 @@ __global__ void __launch_bounds__(XT) skim_exact_kernel(ClusterArgs a, int rows_
             __syncthreads();
             for (int lev = 0; lev < L; ++lev) {
                 const int h = 1 << (L - 1 - lev);
-                const int nodes = 1 << lev;
-                if (nodes <= XT) {
-                    // a group of G threads per node
-                    const int G = XT >> lev;
-                    const int qn = tid / G, r = tid - qn * G;
-                    const int p = (2 * qn + 1) * h;
-                    double best = __longlong_as_double(0x7ff0000000000000ll);     // +inf
-                    int bt = 0x7fffffff;
-                    int i = 0;
-                    if (p <= n) {
-                        i = j + p - 1;
-                        const int tlo = optarr[p - h];
-                        int thi = i - 1;
-                        if (p + h <= n) thi = min(thi, (int)optarr[p + h]);
-                        thi = max(thi, tlo);                   // rounding may break the ordering of two near-tied minimisers
-                        const double4 qi = ld_q(Q + i);
-                        for (int t = tlo + r; t <= thi; t += G) {
-                            const double4 qt = ld_q(Q + t);
-                            const double v = qt.w + interval_cost(qt, qi);
-                            if (v < best) { best = v; bt = t; }
-                        }
+                const int nvalid = (n / h + 1) >> 1;                 // nodes (2q + 1) h <= n of this level
+                // a node's position, and the range of split points its two finished neighbours leave it
+                auto node_i = [&](int q) { return j + (2 * q + 1) * h - 1; };
+                auto node_tlo = [&](int q) { return (int)optarr[2 * q * h]; };
+                auto node_thi = [&](int q) {
+                    const int i = node_i(q);
+                    int thi = i - 1;
+                    if ((2 * q + 2) * h <= n) thi = min(thi, (int)optarr[(2 * q + 2) * h]);
+                    return max(thi, node_tlo(q));                   // rounding may break the order of two near-tied minimisers
+                };
+                for (int q = tid; q < nvalid; q += XT) keys[q] = ~0ull;
+                __syncthreads();
+                // The ranges of a level's nodes tile the span of split points, sharing their end points.  The
+                // span, not the nodes, is dealt to the threads in equal stretches (a node's range can be a
+                // thousand times another's); a thread walks its stretch node by node and commits each node's
+                // best candidate with one atomic minimum on (cost rounded to 2^-36 relative, split point).
+                const int tmin = (int)optarr[0], tmax = node_thi(nvalid - 1);
+                const int chunk = (tmax - tmin + XT) / XT;
+                const int ta = tmin + tid * chunk, tb = min(ta + chunk, tmax + 1);
+                if (ta < tb) {
+                    int lo = 0, hi = nvalid - 1;
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        if (node_thi(mid) < ta) lo = mid + 1; else hi = mid;
                     }
-                    if (G > 1) {
-                        sval[tid] = best;
-                        sarg[tid] = bt;
-                        __syncthreads();
-                        for (int s = G >> 1; s >= 1; s >>= 1) {
-                            if (r < s) {
-                                const double ov = sval[tid + s];
-                                const int ot = sarg[tid + s];
-                                if (ov < best || (ov == best && ot < bt)) { best = ov; bt = ot; }
-                                sval[tid] = best;
-                                sarg[tid] = bt;
+                    for (int q = lo; q < nvalid; ++q) {
+                        const int tlo = node_tlo(q), thi = node_thi(q);
+                        if (tlo >= tb) break;
+                        const int t0 = max(ta, tlo), t1 = min(tb - 1, thi);
+                        if (t0 <= t1) {
+                            const double4 qi = ld_q(Q + node_i(q));
+                            double best = __longlong_as_double(0x7ff0000000000000ll);     // +inf
+                            int bt = t0;
+                            int t = t0;
+                            for (; t + 3 <= t1; t += 4) {            // four loads in flight
+                                const double4 qa = ld_q(Q + t), qb = ld_q(Q + t + 1), qc = ld_q(Q + t + 2), qd = ld_q(Q + t + 3);
+                                const double va = qa.w + interval_cost(qa, qi), vb = qb.w + interval_cost(qb, qi);
+                                const double vc = qc.w + interval_cost(qc, qi), vd = qd.w + interval_cost(qd, qi);
+                                if (va < best) { best = va; bt = t; }
+                                if (vb < best) { best = vb; bt = t + 1; }
+                                if (vc < best) { best = vc; bt = t + 2; }
+                                if (vd < best) { best = vd; bt = t + 3; }
                             }
-                            __syncthreads();
+                            for (; t <= t1; ++t) {
+                                const double4 qt = ld_q(Q + t);
+                                const double v = qt.w + interval_cost(qt, qi);
+                                if (v < best) { best = v; bt = t; }
+                            }
+                            atomicMin(&keys[q], candidate_key(best, bt));
                         }
-                    }
-                    if (r == 0 && p <= n) {
-                        optarr[p] = (uint16_t)bt;
-                        Fc[i] = best;
-                        T[(size_t)j * (m + 1) + i] = (uint16_t)bt;
-                    }
-                } else {
-                    for (int qn = tid; qn < nodes; qn += XT) {
-                        const int p = (2 * qn + 1) * h;
-                        if (p > n) break;
-                        const int i = j + p - 1;
-                        const int tlo = optarr[p - h];
-                        int thi = i - 1;
-                        if (p + h <= n) thi = min(thi, (int)optarr[p + h]);
-                        thi = max(thi, tlo);
-                        const double4 qi = ld_q(Q + i);
-                        double best = __longlong_as_double(0x7ff0000000000000ll);
-                        int bt = tlo;
-                        for (int t = tlo; t <= thi; ++t) {
-                            const double4 qt = ld_q(Q + t);
-                            const double v = qt.w + interval_cost(qt, qi);
-                            if (v < best) { best = v; bt = t; }
-                        }
-                        optarr[p] = (uint16_t)bt;
-                        Fc[i] = best;
-                        T[(size_t)j * (m + 1) + i] = (uint16_t)bt;
+                        if (thi >= tb) break;                        // the rest of this node, and all later ones, are other threads'
                     }
                 }
+                __syncthreads();
+                for (int q = tid; q < nvalid; q += XT) {
+                    const int i = node_i(q);
+                    const double4 qi = ld_q(Q + i);
+                    const unsigned long long key = keys[q];
+                    int bt = (int)(key & 0xffffull);
+                    double best;
+                    if (key != ~0ull) {
+                        const double4 qt = ld_q(Q + bt);
+                        best = qt.w + interval_cost(qt, qi);
+                    } else {
+                        // no stretch met the node (possible only where rounding broke the order of the ranges)
+                        best = __longlong_as_double(0x7ff0000000000000ll);
+                        bt = node_tlo(q);
+                        for (int t = node_tlo(q); t <= node_thi(q); ++t) {
+                            const double4 qt = ld_q(Q + t);
+                            const double v = qt.w + interval_cost(qt, qi);
+                            if (v < best) { best = v; bt = t; }
+                        }
+                    }
+                    Fc[i] = best;
+                    T[(size_t)j * (m + 1) + i] = (uint16_t)bt;
+                }
+                __syncthreads();
+                for (int q = tid; q < nvalid; q += XT) optarr[(2 * q + 1) * h] = T[(size_t)j * (m + 1) + node_i(q)];
                 __syncthreads();
             }
             // F_j becomes the previous layer
@@ -248,12 +282,15 @@ int skim_exact_slots(const skim_ctx *ctx, int64_t rows)
 
 int skim_launch_exact(skim_ctx *ctx, const ClusterArgs &args, int64_t rows, void *scratch, int slots)
 {
-    int L = 1;
-    while ((1 << L) - 1 < args.m) ++L;
-    const size_t smem = ((size_t)(1 << L) + 8) * sizeof(uint16_t);
+    const size_t smem = exact_smem_bytes(args.m);
     if (smem > (size_t)ctx->max_smem_optin) return SKIM_ERR_SHAPE;
     SKIM_CUDA_OK(cudaFuncSetAttribute(skim_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const unsigned blocks = (unsigned)(rows < slots ? rows : slots);
+    // as many blocks as are resident at once (each owns a scratch slot), at most `slots`
+    int per_sm = 1;
+    SKIM_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, skim_exact_kernel, XT, smem));
+    int64_t resident = (int64_t)(per_sm > 0 ? per_sm : 1) * ctx->sm_count;
+    if (resident > slots) resident = slots;
+    const unsigned blocks = (unsigned)(rows < resident ? rows : resident);
     skim_exact_kernel<<<blocks, XT, smem, ctx->stream>>>(args, (int)rows, (unsigned char *)scratch, exact_slot(args.m).total);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
