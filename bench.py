@@ -182,6 +182,33 @@ def run_stage(args, ctx, stream, W, G, cent, bits, out):
                               "algorithmic_bytes_per_step": nbytes, "achieved_gbs": nbytes / (ms * 1e-3) / 1e9,
                               "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
                               "loss_first": float(trace[0]), "loss_last": float(trace[-1]), "kernel_launches_per_step": 3}))
+        elif args.stage == "lfull":
+            tpeak, tpeak_kind = measured_tensor_peak()
+            Hc = torch.from_numpy(inputs.make_gram(COLS, SEED + 7)).cuda()
+            Dbuf = torch.empty((ROWS, COLS), dtype=torch.float16, device="cuda")
+            scr = torch.empty(ctx.err_lfull_bytes(ROWS, COLS), dtype=torch.uint8, device="cuda")
+            col = torch.empty((ROWS,), dtype=torch.float32, device="cuda")
+            ctx.residual(W, cent, BIT_SET, width=BIT_SET[-1], out=Dbuf)
+            for _ in range(2):
+                ctx.err_lfull(Dbuf, Hc, scratch=scr, out=col)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                ctx.err_lfull(Dbuf, Hc, scratch=scr, out=col)
+            e1.record(stream)
+            stream.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            flops = 2.0 * ROWS * COLS * COLS
+            print(json.dumps({"stage": "err_lfull", "workload": WORKLOAD, "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                              "tensor_frac": flops / (ms * 1e-3) / 1e12 / tpeak, "peak_kind": f"of {tpeak_kind}"}))
+        elif args.stage == "exact":
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ctx.cluster_rows_exact(W[:64], G[:64], BIT_SET)
+            e0.record(stream)
+            ctx.cluster_rows_exact(W, G, BIT_SET)
+            e1.record(stream)
+            stream.synchronize()
+            print(json.dumps({"stage": "cluster_rows_exact", "workload": WORKLOAD, "ms": e0.elapsed_time(e1)}))
         else:
             xq = torch.from_numpy(np.random.default_rng(1).standard_normal(COLS).astype(np.float16)).cuda()
             wq = torch.empty((ROWS, COLS), dtype=torch.float16, device="cuda")
@@ -527,9 +554,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--rows", type=int, default=0, help="profiling only: use fewer rows of the same matrix")
-    ap.add_argument("--stage", default="pipeline", choices=["pipeline", "scale", "consumers"],
-                    help="pipeline: the benchmark proper; scale / consumers: time only the alpha-update or the "
-                         "unpacking kernels on the same matrix (their own JSON line; used for profiler captures)")
+    ap.add_argument("--stage", default="pipeline", choices=["pipeline", "scale", "consumers", "lfull", "exact"],
+                    help="pipeline: the benchmark proper; scale / consumers / lfull / exact: time only the alpha-update, the "
+                         "unpacking kernels, the L-full error GEMM or the exact clustering on the same matrix (their own "
+                         "JSON line; used for profiler captures)")
     args = ap.parse_args()
     if args.rows:
         global ROWS, WORKLOAD
