@@ -258,17 +258,20 @@ int skim_launch_cluster(skim_ctx *ctx, const uint16_t *W, const float *importanc
     a.scratch = ws.cluster_scratch;
     a.rec_stride = 0;
     a.row0 = 0;
+    a.rec_half = 0;
     a.early_exit = ctx->early_exit ? 1 : 0;
     a.iter_stats = ctx->timing ? ws.status + 1 : nullptr;
 
     // plan: the fp16-key sort kernel when it applies, else the generic one
-    bool fast = !scaled && skim_launch_sort16(ctx, a, 0, false) == SKIM_OK;
+    // (the exact kernel reads the full records with their g*x^2 prefixes, which only the generic kernel writes)
+    bool fast = !scaled && !exact_scratch && skim_launch_sort16(ctx, a, 0, false) == SKIM_OK;
     const Variant *v = nullptr;
     size_t smem = 0;
     if (!fast) {
         v = pick_variant(scaled ? kVariants32 : kVariants16, cols, ctx->max_smem_optin, &smem);
         if (!v) return SKIM_ERR_SHAPE;
         a.rec_stride = (long long)row_record(a.m).total;
+        a.rec_half = 0;
         SKIM_CUDA_OK(cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
     if ((size_t)a.rec_stride > skim_cluster_record_bytes(cols)) return SKIM_ERR_WORKSPACE;

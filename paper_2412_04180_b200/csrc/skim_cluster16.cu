@@ -326,7 +326,7 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         __syncthreads();
         nd = ps.misc[0];
     }
-    write_row_record<uint16_t, THREADS, false>(a, src, ps, nd, (int)blockIdx.x);
+    write_row_record_half<THREADS>(a, src, ps, nd, (int)blockIdx.x);
     if (nd <= 16) {
         collect_distinct<uint16_t, THREADS>(src, m, nd, ps);
         write_distinct_values(a, nd, ps.dvals, (int)blockIdx.x);
@@ -358,7 +358,8 @@ int skim_launch_sort16(skim_ctx *ctx, ClusterArgs &args, int64_t rows, bool laun
         if (v.cap < cols) continue;
         const Layout16 L = layout16((int)cols, v.threads);
         if (L.total > (size_t)ctx->max_smem_optin) continue;
-        args.rec_stride = (long long)row_record(args.m).total;
+        args.rec_stride = (long long)row_record(args.m, true).total;
+        args.rec_half = 1;
         if (!launch) return SKIM_OK;
         const ClusterArgs a = args;
         // set on every launch: a host-side call of microseconds, and no state shared between contexts

@@ -81,6 +81,7 @@ struct ClusterArgs {
     unsigned char *scratch;   // row records of the current chunk (written by the sort kernel, read by the Lloyd kernel)
     long long rec_stride;     // bytes between row records
     int64_t row0;             // first row of the current chunk
+    int rec_half;             // the records are in the compact format of the fp16-key sort kernel
     int early_exit;           // stop a row once no boundary moved
     unsigned long long *iter_stats;   // nullptr, or two counters: iterations run, rows counted
 };
@@ -103,12 +104,18 @@ struct RowRecord {
     int ngrp, nseg;
 };
 constexpr int SKIM_GROUP_BYTES = 96;                // three 32-byte sectors
+// Compact record of the fp16-key sort kernel (no scale installed, so a value IS a binary16 number): a group is
+// two sectors, 8 binary16 values | the binary64 sums of g and g*x from the segment start | the 8 importances.
+// The g*x^2 sums are not kept per group: the error of a width is  sum g x^2 (row total, last segment entry)
+// minus  sum_j c_j (2 S1_j - c_j S0_j),  which needs the interval sums of g and g*x only.
+constexpr int SKIM_GROUP_BYTES_HALF = 64;
+constexpr unsigned short SKIM_PAD_HALF = 0x7bffu;   // largest finite binary16
 constexpr int SKIM_SEG_SHIFT = 5;                   // a segment is 32 groups (256 elements): one group per lane of a warp
 constexpr float SKIM_PAD_VALUE = 3.402823466e38f;   // largest finite binary32: 0 * padding stays 0
 
 __host__ __device__ inline int sk_entries(int m) { return ((((m + 7) >> 3) + 7) & ~7) + 16; }
 
-__host__ __device__ inline RowRecord row_record(int m)
+__host__ __device__ inline RowRecord row_record(int m, bool half_groups = false)
 {
     RowRecord R;
     R.ngrp = (m + 7) >> 3;
@@ -116,7 +123,7 @@ __host__ __device__ inline RowRecord row_record(int m)
     R.gi_bytes = (size_t)sk_entries(m) * 4;
     size_t off = 128;
     R.seg = off; off += (size_t)(R.nseg + 1) * 32;
-    R.groups = off; off += (size_t)R.ngrp * SKIM_GROUP_BYTES;
+    R.groups = off; off += (size_t)R.ngrp * (half_groups ? SKIM_GROUP_BYTES_HALF : SKIM_GROUP_BYTES);
     R.gi = off; off += R.gi_bytes;
     R.total = (off + 127) & ~(size_t)127;
     return R;
@@ -164,6 +171,7 @@ template <typename KeyT> struct SortedArrays {
 // Small per-block scratch of the phases below.
 struct PhaseSmem {
     double segtot[96][3];   // sums of every segment (rows of up to 24 576 elements have 96 segments of 32 groups)
+    double wsum2[32];       // compact record: every warp's sum of g*x^2
     float tfs[32];     // scratch of collect_distinct
     float dvals[32];   // the row's distinct values when there are at most 16
     int misc[4];       // [0] distinct count, [1] slot counter
@@ -328,6 +336,121 @@ __device__ __forceinline__ int write_row_record(const ClusterArgs &a, const Src 
         if (lane == 0) *reinterpret_cast<int *>(rec) = nd;
     }
     return nd;
+}
+
+// One 32-byte store of four 64-bit words.
+__device__ __forceinline__ void st_sector(void *p, unsigned long long a, unsigned long long b, unsigned long long c, unsigned long long d)
+{
+    asm volatile("st.global.v4.b64 [%0], {%1, %2, %3, %4};" ::"l"(p), "l"(a), "l"(b), "l"(c), "l"(d) : "memory");
+}
+
+// The compact row record (see SKIM_GROUP_BYTES_HALF) from a row sorted by 16-bit keys; the counterpart of
+// write_row_record for the fp16-key sort kernel.  One pass, one group per lane; only the sums of g and g*x are
+// scanned, the g*x^2 terms are added up per warp and meet in the row total.  nd: the distinct-value count
+// (any number above 16 stands for "more than 16").  Call with all threads.
+template <int THREADS, typename Src>
+__device__ __forceinline__ void write_row_record_half(const ClusterArgs &a, const Src &src, PhaseSmem &ps, int nd, int local_row)
+{
+    constexpr int NW = THREADS / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int m = a.m;
+    const RowRecord R = row_record(m, true);
+    unsigned char *rec = a.scratch + (size_t)local_row * (size_t)a.rec_stride;
+    float *gi = reinterpret_cast<float *>(rec + R.gi);
+    unsigned bad = 0u;
+    double w2acc = 0.0;
+    for (int sgm = warp; sgm < R.nseg; sgm += NW) {
+        const int q = (sgm << SKIM_SEG_SHIFT) + lane;
+        double v0 = 0.0, v1 = 0.0;
+        unsigned long long xq0 = 0ull, xq1 = 0ull;
+        float first = 0.0f;
+        if (q < R.ngrp) {
+            const int e = q << 3;
+            uint16_t ks[8];
+            float gs[8];
+            const unsigned gbits = src.group(e, m, ks, gs);
+            uint32_t hb[8];
+            double xd[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint16_t k = ks[u];
+                const uint16_t h = (e + u < m) ? ((k & 0x8000u) ? (uint16_t)(k & 0x7fffu) : (uint16_t)~k) : (uint16_t)SKIM_PAD_HALF;
+                hb[u] = h;
+                xd[u] = (double)__half2float(__ushort_as_half(h));
+            }
+            xq0 = (unsigned long long)(hb[0] | (hb[1] << 16)) | ((unsigned long long)(hb[2] | (hb[3] << 16)) << 32);
+            xq1 = (unsigned long long)(hb[4] | (hb[5] << 16)) | ((unsigned long long)(hb[6] | (hb[7] << 16)) << 32);
+            first = (float)xd[0];
+            st_sector(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES_HALF + 32, gs);
+            double t0[8], t1[8], t2[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const double g = (double)gs[u];                       // padding: g = 0, x finite
+                t0[u] = g;
+                t1[u] = g * xd[u];
+                t2[u] = t1[u] * xd[u];
+            }
+            v0 = ((t0[0] + t0[1]) + (t0[2] + t0[3])) + ((t0[4] + t0[5]) + (t0[6] + t0[7]));
+            v1 = ((t1[0] + t1[1]) + (t1[2] + t1[3])) + ((t1[4] + t1[5]) + (t1[6] + t1[7]));
+            w2acc += ((t2[0] + t2[1]) + (t2[2] + t2[3])) + ((t2[4] + t2[5]) + (t2[6] + t2[7]));
+            if ((gbits >> 31) || !(v0 < 1.0e300)) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (!(gs[u] >= 0.0f) || gs[u] > 3.0e38f) bad |= 2u;
+            }
+        }
+        double i0 = v0, i1 = v1;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const double u0 = __shfl_up_sync(0xffffffffu, i0, off);
+            const double u1 = __shfl_up_sync(0xffffffffu, i1, off);
+            if (lane >= off) { i0 += u0; i1 += u1; }
+        }
+        if (lane == 31 && SKIM_IDX(sgm, 96, a.status)) { ps.segtot[sgm][0] = i0; ps.segtot[sgm][1] = i1; }
+        double e0 = __shfl_up_sync(0xffffffffu, i0, 1), e1 = __shfl_up_sync(0xffffffffu, i1, 1);
+        if (lane == 0) { e0 = 0.0; e1 = 0.0; }
+        if (q < R.ngrp) {
+            st_sector(rec + R.groups + (size_t)q * SKIM_GROUP_BYTES_HALF, xq0, xq1,
+                      (unsigned long long)__double_as_longlong(e0), (unsigned long long)__double_as_longlong(e1));
+            gi[q] = first;
+        }
+    }
+    if (bad) atomicOr(a.status, (unsigned long long)bad);
+    for (int q = R.ngrp + threadIdx.x; q < sk_entries(m); q += THREADS) gi[q] = SKIM_PAD_VALUE;
+    // every warp's sum of g*x^2, lanes added in a fixed order
+#pragma unroll
+    for (int off = 16; off; off >>= 1) w2acc += __shfl_xor_sync(0xffffffffu, w2acc, off);
+    if (lane == 0) ps.wsum2[warp] = w2acc;
+    __syncthreads();
+    if (warp == 0) {
+        double run0 = 0.0, run1 = 0.0, loc[4][2];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int sgm = lane * 4 + u;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) loc[u][c] = sgm < R.nseg ? ps.segtot[sgm][c] : 0.0;
+            run0 += loc[u][0]; run1 += loc[u][1];
+        }
+        double i0 = run0, i1 = run1;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const double u0 = __shfl_up_sync(0xffffffffu, i0, off);
+            const double u1 = __shfl_up_sync(0xffffffffu, i1, off);
+            if (lane >= off) { i0 += u0; i1 += u1; }
+        }
+        double b0 = __shfl_up_sync(0xffffffffu, i0, 1), b1 = __shfl_up_sync(0xffffffffu, i1, 1);
+        if (lane == 0) { b0 = 0.0; b1 = 0.0; }
+        double s2 = 0.0;
+        for (int w = 0; w < NW; ++w) s2 += ps.wsum2[w];
+        double4 *seg = reinterpret_cast<double4 *>(rec + R.seg);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int sgm = lane * 4 + u;
+            if (sgm <= R.nseg) seg[sgm] = make_double4(b0, b1, sgm == R.nseg ? s2 : 0.0, 0.0);   // entry nseg: the row totals
+            b0 += loc[u][0]; b1 += loc[u][1];
+        }
+        if (lane == 0) *reinterpret_cast<int *>(rec) = nd;
+    }
 }
 
 // Stores the row's distinct values (nd <= 16 of them, from collect_distinct) in the record header.

@@ -32,8 +32,13 @@ __device__ __forceinline__ void ld_sector(const unsigned char *p, float4 &a, flo
                  : "l"(p));
 }
 
-// One group record in registers.
-struct Group {
+// One group record in registers.  HALF = false: the full record (three sectors: binary32 values | importances |
+// sums incl. g*x^2); HALF = true: the compact record of the fp16-key sort kernel (two sectors: binary16 values
+// and the sums of g and g*x | importances).
+template <bool HALF> struct Group;
+
+template <> struct Group<false> {
+    static constexpr int BYTES = SKIM_GROUP_BYTES;
     float4 xa, xb, ga, gb;
     double2 p;   // prefix sums of g and g*x at the group's first element
     __device__ __forceinline__ void load(const unsigned char *gr)
@@ -48,20 +53,68 @@ struct Group {
     {
         return (xa.x <= t) + (xa.y <= t) + (xa.z <= t) + (xa.w <= t) + (xb.x <= t) + (xb.y <= t) + (xb.z <= t) + (xb.w <= t);
     }
+    __device__ __forceinline__ void values(double *x) const
+    {
+        x[0] = (double)xa.x; x[1] = (double)xa.y; x[2] = (double)xa.z; x[3] = (double)xa.w;
+        x[4] = (double)xb.x; x[5] = (double)xb.y; x[6] = (double)xb.z; x[7] = (double)xb.w;
+    }
+    static __device__ __forceinline__ float value_at(const unsigned char *groups, int idx)
+    {
+        return __ldg(reinterpret_cast<const float *>(groups + (size_t)(idx >> 3) * BYTES) + (idx & 7));
+    }
+};
+
+template <> struct Group<true> {
+    static constexpr int BYTES = SKIM_GROUP_BYTES_HALF;
+    uint32_t xh[4];      // 8 binary16 values
+    float4 ga, gb;
+    double2 p;
+    __device__ __forceinline__ void load(const unsigned char *gr)
+    {
+        unsigned long long q0, q1, q2, q3;
+        asm volatile("ld.global.nc.v4.b64 {%0, %1, %2, %3}, [%4];" : "=l"(q0), "=l"(q1), "=l"(q2), "=l"(q3) : "l"(gr));
+        xh[0] = (uint32_t)q0; xh[1] = (uint32_t)(q0 >> 32); xh[2] = (uint32_t)q1; xh[3] = (uint32_t)(q1 >> 32);
+        p = make_double2(__longlong_as_double((long long)q2), __longlong_as_double((long long)q3));
+        ld_sector(gr + 32, ga, gb);
+    }
+    // a binary16 value is <= t exactly when it is <= t rounded down to binary16: four packed compares
+    __device__ __forceinline__ int count_le(float t) const
+    {
+        const __half2 th = __half2half2(__float2half_rd(t));
+        __half2 c = __hle2(*reinterpret_cast<const __half2 *>(&xh[0]), th);
+        c = __hadd2(c, __hle2(*reinterpret_cast<const __half2 *>(&xh[1]), th));
+        c = __hadd2(c, __hle2(*reinterpret_cast<const __half2 *>(&xh[2]), th));
+        c = __hadd2(c, __hle2(*reinterpret_cast<const __half2 *>(&xh[3]), th));
+        return (int)(__low2float(c) + __high2float(c));
+    }
+    __device__ __forceinline__ void values(double *x) const
+    {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&xh[u]));
+            x[2 * u] = (double)f.x;
+            x[2 * u + 1] = (double)f.y;
+        }
+    }
+    static __device__ __forceinline__ float value_at(const unsigned char *groups, int idx)
+    {
+        return __half2float(__ushort_as_half(__ldg(reinterpret_cast<const unsigned short *>(groups + (size_t)(idx >> 3) * BYTES) + (idx & 7))));
+    }
 };
 
 // Adds the first n (0..8) elements of a group to (s0, s1[, s2]): the eight terms are summed pairwise,
 // a fixed order with a short dependency chain.  Elements past n are masked before any arithmetic.
-template <bool WANT_C>
-__device__ __forceinline__ void add_group(const Group &grp, int n, double &s0, double &s1, double &s2)
+template <bool WANT_C, typename G>
+__device__ __forceinline__ void add_group(const G &grp, int n, double &s0, double &s1, double &s2)
 {
-    const float xs[8] = {grp.xa.x, grp.xa.y, grp.xa.z, grp.xa.w, grp.xb.x, grp.xb.y, grp.xb.z, grp.xb.w};
+    double xs[8];
+    grp.values(xs);
     const float gs[8] = {grp.ga.x, grp.ga.y, grp.ga.z, grp.ga.w, grp.gb.x, grp.gb.y, grp.gb.z, grp.gb.w};
     double t0[8], t1[8], t2[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
         const bool in = u < n;
-        const double g = (double)(in ? gs[u] : 0.0f), x = (double)xs[u];   // padding values are finite, so 0 * x = 0
+        const double g = (double)(in ? gs[u] : 0.0f), x = xs[u];   // padding values are finite, so 0 * x = 0
         t0[u] = g;
         t1[u] = g * x;
         if (WANT_C) t2[u] = t1[u] * x;
@@ -123,12 +176,13 @@ __device__ __forceinline__ double quotient(double s1, double s0)
 // window); loads that one group record, which gives the exact boundary position (values), the
 // prefix sums at the group start and the few elements in between.
 // On return sm.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
+template <bool HALF>
 __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float *gi, int nd, const ClusterArgs &a, int64_t row,
                                            LloydSmem &sm)
 {
     const int lane = threadIdx.x & 31;
     const int m = a.m;
-    const RowRecord R = row_record(m);
+    const RowRecord R = row_record(m, HALF);
     const unsigned char *groups = rec + R.groups;
     const double4 *seg = reinterpret_cast<const double4 *>(rec + R.seg);   // 32-byte entries; a few hot lines, served by L1
     const int ngi = sk_entries(m) - 16;                 // group-index entries up to the padding margin
@@ -148,8 +202,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
     if (degenerate) c = sm.dvals[min(j, nd - 1)];
     if (normal) {
         const int idx = (int)(((long long)(2 * j + 1) * m) / (2 * k));
-        if (SKIM_IDX(idx, m, a.status))
-            c = __ldg(reinterpret_cast<const float *>(groups + (size_t)(idx >> 3) * SKIM_GROUP_BYTES) + (idx & 7));
+        if (SKIM_IDX(idx, m, a.status)) c = Group<HALF>::value_at(groups, idx);
     }
 
     int Bprev = -1;
@@ -160,7 +213,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
     for (int it = 0;; ++it) {
         const float c_up = __shfl_down_sync(0xffffffffu, c, 1);
         int B = m, grp_i = 0, cntk = 0;
-        Group grp;
+        Group<HALF> grp;
         if (has_boundary) {
             // exact midpoint of two binary32 centroids, rounded down to binary32: x <= midpoint
             // holds for a binary32 x exactly when x <= tf
@@ -187,7 +240,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
             if (!SKIM_IDX(grp_i, R.ngrp, a.status)) grp_i = 0;
             gstep = gprev >= 0 ? grp_i - gprev : 0;
             gprev = grp_i;
-            const unsigned char *gr = groups + (size_t)grp_i * SKIM_GROUP_BYTES;
+            const unsigned char *gr = groups + (size_t)grp_i * Group<HALF>::BYTES;
             grp.load(gr);
             cntk = grp.count_le(tf);
             B = min((grp_i << 3) + cntk, m);
@@ -201,7 +254,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 const double2 sb = __ldg(reinterpret_cast<const double2 *>(seg + (grp_i >> SKIM_SEG_SHIFT)));   // sums of the earlier segments
                 P0 = sb.x + grp.p.x;
                 P1 = sb.y + grp.p.y;
-                if (final) {
+                if (final && !HALF) {
                     Pc = __ldg(&seg[grp_i >> SKIM_SEG_SHIFT].z) + __ldg(reinterpret_cast<const double *>(groups + (size_t)grp_i * SKIM_GROUP_BYTES + 80));
                     add_group<true>(grp, cntk, P0, P1, Pc);
                 } else {
@@ -212,18 +265,20 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 const double2 tot = __ldg(reinterpret_cast<const double2 *>(seg + R.nseg));
                 P0 = tot.x;
                 P1 = tot.y;
-                if (final) Pc = __ldg(&seg[R.nseg].z);
+                if (final && !HALF) Pc = __ldg(&seg[R.nseg].z);
             }
         }
         double Q0 = __shfl_up_sync(0xffffffffu, P0, 1);
         double Q1 = __shfl_up_sync(0xffffffffu, P1, 1);
-        double Qc = final ? __shfl_up_sync(0xffffffffu, Pc, 1) : 0.0;
+        double Qc = (final && !HALF) ? __shfl_up_sync(0xffffffffu, Pc, 1) : 0.0;
         if (j == 0) { Q0 = 0.0; Q1 = 0.0; Qc = 0.0; }
         const double S0 = P0 - Q0, S1 = P1 - Q1;
         if (final) {
             if (normal) {
                 const double cd = (double)c, S2 = Pc - Qc;
-                err_j = fmax(fma(cd, fma(cd, S0, -2.0 * S1), S2), 0.0);
+                // full record: the cluster's own error; compact record: the part the row total of g*x^2 is
+                // reduced by, c (2 S1 - c S0)
+                err_j = HALF ? cd * fma(-cd, S0, 2.0 * S1) : fmax(fma(cd, fma(cd, S0, -2.0 * S1), S2), 0.0);
             }
             if (a.iter_stats && lane == 0) {
                 atomicAdd(a.iter_stats, (unsigned long long)it);       // assign/update pairs this row ran
@@ -244,6 +299,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
         if (j == 0 && a.err) {
             double e = 0.0;
             for (int u = 0; u < k; ++u) e += sm.errs[lane + u];
+            if (HALF) e = normal ? fmax(__ldg(&reinterpret_cast<const double4 *>(rec + R.seg)[R.nseg].z) - e, 0.0) : 0.0;
             if (a.row_bits) a.err[row] = (float)e; else a.err[row * a.nb + bi] = (float)e;
         }
     }
@@ -273,6 +329,7 @@ __device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, c
     }
 }
 
+template <bool HALF>
 __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(ClusterArgs a, int rows_in_chunk)
 {
     __shared__ LloydSmem sm_all[LLOYD_WARPS];
@@ -291,12 +348,12 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
     const int nsk = sk_entries(a.m);
     float *gi = gi_all + (size_t)warp * nsk;
     {
-        const float4 *src = reinterpret_cast<const float4 *>(rec + row_record(a.m).gi);
+        const float4 *src = reinterpret_cast<const float4 *>(rec + row_record(a.m, HALF).gi);
         float4 *dst = reinterpret_cast<float4 *>(gi);
         for (int i = lane; i < nsk / 4; i += 32) dst[i] = __ldg(src + i);
     }
     __syncwarp();
-    lloyd_warp(rec, gi, nd, a, row, sm);
+    lloyd_warp<HALF>(rec, gi, nd, a, row, sm);
     if (!a.codes) return;
     __syncwarp();
     write_codes(a, row, sm);
@@ -309,8 +366,9 @@ int skim_launch_lloyd(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
     const unsigned blocks = (unsigned)((rows + LLOYD_WARPS - 1) / LLOYD_WARPS);
     const size_t smem = (size_t)LLOYD_WARPS * sk_entries(args.m) * sizeof(float);
     // set on every launch: a host-side call of microseconds, and no state shared between contexts
-    SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lloyd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    skim_lloyd_kernel<<<blocks, LLOYD_WARPS * 32, smem, ctx->stream>>>(args, (int)rows);
+    void (*kernel)(ClusterArgs, int) = args.rec_half ? skim_lloyd_kernel<true> : skim_lloyd_kernel<false>;
+    SKIM_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<blocks, LLOYD_WARPS * 32, smem, ctx->stream>>>(args, (int)rows);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     return SKIM_OK;
