@@ -869,6 +869,105 @@ int skim_oracle_err_lfull(const uint16_t *D, int64_t rows, int64_t cols, int64_t
     return failed ? -4 : 0;
 }
 
+/*
+ * Loss and gradient of the scaling vector in the L-full form (Section 4.3: "the loss calculation adopts the L-full
+ * form"; Algorithm 2, inner repeat; Section 3.4 for the form itself), labels fixed:
+ *     c_ik  = sum_{j in k} g_ij W_ij / alpha_j  /  sum_{j in k} g_ij     (importance-weighted, as in the diagonal version)
+ *     d_ij  = W_ij - alpha_j c_{i,l_ij}
+ *     loss  = sum_i d_i H d_i^T,   H = X X^T (binary16, symmetric)
+ * With Y = D H the derivative with respect to d_ij is 2 Y_ij, so, both through the explicit alpha_j and through the
+ * re-fitted centroids,
+ *     d loss / d alpha_j = sum_i [ -2 Y_ij c_{i,l_ij} + 2 R_{i,l_ij} g_ij W_ij / (alpha_j^2 G_{i,l_ij}) ],
+ *     R_ik = sum_{j in k} Y_ij alpha_j,   G_ik = sum_{j in k} g_ij.
+ * round_d != 0: the residual enters the contraction as the library's operand does, binary16(float(d) * 2^exp2) / 2^exp2
+ * (the gradient treats that rounding as the identity); round_d == 0: exact d (used by the finite-difference pin).
+ *   grad out [cols], may be NULL.
+ */
+int skim_oracle_scale_loss_grad_lfull(const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                                      int64_t ld, const uint8_t *labels, const double *alpha, const uint16_t *H,
+                                      int64_t ldh, int exp2, int round_d, double *loss_out, double *grad)
+{
+    if (!W || !importance || !labels || !alpha || !H || rows <= 0 || cols <= 0 || ld < cols || ldh < cols) return -1;
+    double *Hd = (double *)malloc((size_t)cols * (size_t)cols * sizeof(double));
+    double *rowbuf = (double *)malloc((size_t)cols * 2 * sizeof(double));
+    if (!Hd || !rowbuf) { free(Hd); free(rowbuf); return -1; }
+    for (int64_t j = 0; j < cols; ++j)
+        for (int64_t k = 0; k < cols; ++k) Hd[j * cols + k] = (double)half_bits_to_float(H[j * ldh + k]);
+    double *d = rowbuf, *y = rowbuf + cols;
+    double loss = 0.0;
+    if (grad) for (int64_t j = 0; j < cols; ++j) grad[j] = 0.0;
+    for (int64_t i = 0; i < rows; ++i) {
+        double G[SKIM_ORACLE_MAX_K], S[SKIM_ORACLE_MAX_K], c[SKIM_ORACLE_MAX_K], R[SKIM_ORACLE_MAX_K];
+        for (int k = 0; k < SKIM_ORACLE_MAX_K; ++k) { G[k] = 0.0; S[k] = 0.0; c[k] = 0.0; R[k] = 0.0; }
+        for (int64_t j = 0; j < cols; ++j) {
+            double w = (double)half_bits_to_float(W[i * ld + j]);
+            double g = (double)importance[i * ld + j];
+            int l = labels[i * cols + j];
+            G[l] += g;
+            S[l] += g * w / alpha[j];
+        }
+        for (int k = 0; k < SKIM_ORACLE_MAX_K; ++k) if (G[k] > 0.0) c[k] = S[k] / G[k];
+        for (int64_t j = 0; j < cols; ++j) {
+            double w = (double)half_bits_to_float(W[i * ld + j]);
+            double r = w - alpha[j] * c[labels[i * cols + j]];
+            if (round_d) r = ldexp((double)half_bits_to_float(float_to_half_bits(ldexpf((float)r, exp2))), -exp2);
+            d[j] = r;
+        }
+        for (int64_t k = 0; k < cols; ++k) {
+            double acc = 0.0;
+            for (int64_t j = 0; j < cols; ++j) acc += d[j] * Hd[j * cols + k];
+            y[k] = acc;
+        }
+        for (int64_t j = 0; j < cols; ++j) {
+            loss += y[j] * d[j];
+            R[labels[i * cols + j]] += y[j] * alpha[j];
+        }
+        if (grad) {
+            for (int64_t j = 0; j < cols; ++j) {
+                double w = (double)half_bits_to_float(W[i * ld + j]);
+                double g = (double)importance[i * ld + j];
+                int l = labels[i * cols + j];
+                double t = -2.0 * y[j] * c[l];
+                if (G[l] > 0.0) t += 2.0 * R[l] * g * w / (alpha[j] * alpha[j] * G[l]);
+                grad[j] += t;
+            }
+        }
+    }
+    free(Hd); free(rowbuf);
+    *loss_out = loss;
+    return 0;
+}
+
+/* `steps` Adam updates of alpha on the L-full loss (schedule and constants as in skim_oracle_scale_update). */
+int skim_oracle_scale_update_lfull(const uint16_t *W, const float *importance, int64_t rows, int64_t cols, int64_t ld,
+                                   const uint8_t *labels, const uint16_t *H, int64_t ldh, int exp2, int round_d,
+                                   double *alpha, int steps, double lr0, double decay, int decay_every, double beta1,
+                                   double beta2, double eps, double *loss_trace)
+{
+    if (steps < 0 || decay_every <= 0) return -1;
+    double *m1 = (double *)calloc((size_t)cols, sizeof(double));
+    double *m2 = (double *)calloc((size_t)cols, sizeof(double));
+    double *grad = (double *)malloc((size_t)cols * sizeof(double));
+    if (!m1 || !m2 || !grad) { free(m1); free(m2); free(grad); return -1; }
+    int rc = 0;
+    for (int t = 0; t < steps && !rc; ++t) {
+        double loss;
+        rc = skim_oracle_scale_loss_grad_lfull(W, importance, rows, cols, ld, labels, alpha, H, ldh, exp2, round_d, &loss, grad);
+        if (loss_trace) loss_trace[t] = loss;
+        double lr = lr0 * pow(decay, (double)(t / decay_every));
+        double bc1 = 1.0 - pow(beta1, (double)(t + 1));
+        double bc2 = 1.0 - pow(beta2, (double)(t + 1));
+        for (int64_t j = 0; j < cols; ++j) {
+            m1[j] = beta1 * m1[j] + (1.0 - beta1) * grad[j];
+            m2[j] = beta2 * m2[j] + (1.0 - beta2) * grad[j] * grad[j];
+            double mh = m1[j] / bc1, vh = m2[j] / bc2;
+            alpha[j] -= lr * mh / (sqrt(vh) + eps);
+        }
+    }
+    free(m1); free(m2); free(grad);
+    return rc;
+}
+
 int skim_oracle_num_threads(void)
 {
 #ifdef _OPENMP

@@ -299,6 +299,46 @@ def scale_loss_grad(W, importance, labels, alpha, want_grad=True):
     return loss.value, grad
 
 
+def scale_loss_grad_lfull(W, importance, labels, alpha, H, exp2=8, round_d=True, want_grad=True):
+    """L-full loss sum_i d_i H d_i^T of the scaling vector and its gradient (labels fixed)."""
+    W = np.ascontiguousarray(W)
+    H = np.ascontiguousarray(H)
+    assert W.dtype == np.float16 and H.dtype == np.float16
+    importance = np.ascontiguousarray(importance, dtype=np.float32)
+    labels = np.ascontiguousarray(labels, dtype=np.uint8)
+    alpha = np.ascontiguousarray(alpha, dtype=np.float64)
+    rows, cols = W.shape
+    loss = C.c_double(0.0)
+    grad = np.zeros(cols, dtype=np.float64) if want_grad else None
+    rc = lib().skim_oracle_scale_loss_grad_lfull(_p(W.view(np.uint16)), _p(importance), C.c_int64(rows), C.c_int64(cols),
+                                                 C.c_int64(cols), _p(labels), _p(alpha), _p(H.view(np.uint16)), C.c_int64(cols),
+                                                 C.c_int(exp2), C.c_int(1 if round_d else 0), C.byref(loss), _p(grad))
+    if rc:
+        raise ValueError(f"skim_oracle_scale_loss_grad_lfull failed ({rc})")
+    return loss.value, grad
+
+
+def scale_update_lfull(W, importance, labels, alpha, H, steps=120, exp2=8, round_d=True, lr0=0.01, decay=0.5,
+                       decay_every=40, beta1=0.9, beta2=0.999, eps=1e-8):
+    """Returns (alpha float64 [cols] after `steps` Adam steps on the L-full loss, loss trace [steps])."""
+    W = np.ascontiguousarray(W)
+    H = np.ascontiguousarray(H)
+    assert W.dtype == np.float16 and H.dtype == np.float16
+    importance = np.ascontiguousarray(importance, dtype=np.float32)
+    labels = np.ascontiguousarray(labels, dtype=np.uint8)
+    alpha = np.array(alpha, dtype=np.float64, copy=True)
+    rows, cols = W.shape
+    trace = np.zeros(steps, dtype=np.float64)
+    rc = lib().skim_oracle_scale_update_lfull(_p(W.view(np.uint16)), _p(importance), C.c_int64(rows), C.c_int64(cols),
+                                              C.c_int64(cols), _p(labels), _p(H.view(np.uint16)), C.c_int64(cols),
+                                              C.c_int(exp2), C.c_int(1 if round_d else 0), _p(alpha), C.c_int(steps),
+                                              C.c_double(lr0), C.c_double(decay), C.c_int(decay_every), C.c_double(beta1),
+                                              C.c_double(beta2), C.c_double(eps), _p(trace))
+    if rc:
+        raise ValueError(f"skim_oracle_scale_update_lfull failed ({rc})")
+    return alpha, trace
+
+
 def scale_update(W, importance, labels, alpha, steps=120, lr0=0.01, decay=0.5, decay_every=40,
                  beta1=0.9, beta2=0.999, eps=1e-8):
     """Returns (alpha float64 [cols] after `steps` Adam steps, loss trace [steps])."""

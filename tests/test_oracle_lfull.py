@@ -112,3 +112,69 @@ def test_lfull_error_decreases_with_the_width_on_the_synthetic_gram(oracle):
     table = np.stack([oracle.err_lfull(oracle.residual(w, c32, BITS, width=b), H)[0] for b in BITS], axis=1)
     assert np.all(table >= 0)
     assert np.mean(table[:, 0] > table[:, 3]) == 1.0
+
+
+def _labels_for(oracle, w, g, bits):
+    res = oracle.cluster_rows(w, g, BITS, 15, row_bits=bits)
+    return np.stack([res["codes"][int(b) - 1, i] for i, b in enumerate(bits)]).astype(np.uint8)
+
+
+def test_scale_lfull_gradient_equals_finite_differences(oracle):
+    """The analytic gradient of the L-full loss of the scaling vector (both terms: the explicit alpha and the
+    re-fitted centroids) against central differences of the loss itself, on exact residuals."""
+    rows, cols = 6, 40
+    w, g = inputs.make_rows(rows, cols, 71, outlier_frac=0.02)
+    bits = (np.arange(rows) % 4 + 1).astype(np.uint8)
+    labels = _labels_for(oracle, w, g, bits)
+    H = inputs.make_gram(cols, 72)
+    alpha = inputs.make_scale(cols, 73, spread=0.1).astype(np.float64)
+    loss, grad = oracle.scale_loss_grad_lfull(w, g, labels, alpha, H, round_d=False)
+    # the loss itself, independently: rows of D from numpy, quadratic form by matrix products
+    x = w.astype(np.float64)
+    D = np.zeros_like(x)
+    for i in range(rows):
+        for k in range(16):
+            sel = labels[i] == k
+            if sel.any() and g[i, sel].sum() > 0:
+                c = np.sum(g[i, sel] * x[i, sel] / alpha[sel]) / np.sum(g[i, sel].astype(np.float64))
+                D[i, sel] = x[i, sel] - alpha[sel] * c
+    Hd = H.astype(np.float64)
+    assert loss == pytest.approx(np.einsum("ij,jk,ik->", D, Hd, D), rel=1e-12)
+    for j in (0, 7, 19, 39):
+        h = 1e-6 * alpha[j]
+        ap, am = alpha.copy(), alpha.copy()
+        ap[j] += h
+        am[j] -= h
+        fd = (oracle.scale_loss_grad_lfull(w, g, labels, ap, H, round_d=False, want_grad=False)[0]
+              - oracle.scale_loss_grad_lfull(w, g, labels, am, H, round_d=False, want_grad=False)[0]) / (2 * h)
+        assert grad[j] == pytest.approx(fd, rel=2e-5, abs=1e-9 * np.abs(grad).max())
+
+
+def test_scale_lfull_with_diagonal_h_is_the_diagonal_update(oracle):
+    """H = diag(h) and importance h down every column: the L-full loss of the scaling vector IS the diagonal one,
+    so loss trace and alpha of the two oracle routines agree step for step."""
+    rows, cols, steps = 10, 96, 25
+    w, _ = inputs.make_rows(rows, cols, 81)
+    h = np.exp(0.5 * np.random.default_rng(82).standard_normal(cols)).astype(np.float16)
+    g = np.tile(h.astype(np.float32), (rows, 1))
+    bits = (np.arange(rows) % 4 + 1).astype(np.uint8)
+    labels = _labels_for(oracle, w, g, bits)
+    H = np.diag(h.astype(np.float64)).astype(np.float16)
+    a0 = np.ones(cols)
+    a_diag, t_diag = oracle.scale_update(w, g, labels, a0, steps=steps)
+    a_full, t_full = oracle.scale_update_lfull(w, g, labels, a0, H, steps=steps, round_d=False)
+    np.testing.assert_allclose(t_full, t_diag, rtol=1e-10)
+    np.testing.assert_allclose(a_full, a_diag, rtol=1e-9)
+    # with the binary16 residual operand the loss moves by its rounding (2^-11 per element) and no more
+    _, t_round = oracle.scale_update_lfull(w, g, labels, a0, H, steps=steps, round_d=True)
+    np.testing.assert_allclose(t_round, t_diag, rtol=2e-3)
+
+
+def test_scale_lfull_training_lowers_the_loss(oracle):
+    rows, cols = 24, 64
+    w, g = inputs.make_rows(rows, cols, 91)
+    bits = np.full(rows, 3, np.uint8)
+    labels = _labels_for(oracle, w, g, bits)
+    H = inputs.make_gram(cols, 92)
+    _, trace = oracle.scale_update_lfull(w, g, labels, np.ones(cols), H, steps=40)
+    assert trace[-1] < trace[0]
