@@ -54,6 +54,16 @@ def measured_peak():
         return 6650.0, "fallback"
 
 
+def ctypes_size(ctx, rows, cols):
+    """Scratch bytes of the L-full alpha-update (skim_scale_lfull_bytes)."""
+    import ctypes as C
+    from paper_2412_04180_b200 import skim
+    need = C.c_size_t()
+    rc = skim.lib().skim_scale_lfull_bytes(C.c_int64(rows), C.c_int64(cols), C.byref(need))
+    assert rc == 0
+    return need.value
+
+
 def measured_tensor_peak():
     """Measured dense bf16 tensor throughput (TFLOP/s) for a kernel timed alone; fp16 runs at the same rate."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -420,13 +430,30 @@ def run_ours(args):
                 res_ms += l0.elapsed_time(l1)
                 gemm_ms += l1.elapsed_time(l2)
             assert ctx.get_status() == 0 and bool(torch.isfinite(table).all())
+            # the alpha-update on the L-full loss (Section 4.3): residual, contraction with Y kept, two streaming passes, Adam
+            ctx.apply_scale(None)
+            _, labels0, _ = ctx.cluster_rows_at(W, G, bits, BIT_SET, ITERS, want_codes=True, centroids=cent.clone())
+            alpha_lf = torch.ones(COLS, dtype=torch.float32, device="cuda")
+            need_lf = ctypes_size(ctx, ROWS, COLS)
+            scr_lf = torch.empty(need_lf, dtype=torch.uint8, device="cuda")
+            ctx.scale_update_lfull(W, G, labels0, alpha_lf, Hc, steps=2, want_trace=False, scratch=scr_lf)
+            l0.record(stream)
+            tr = ctx.scale_update_lfull(W, G, labels0, alpha_lf, Hc, steps=10, scratch=scr_lf)
+            l1.record(stream)
+            stream.synchronize()
+            lf_step_ms = l0.elapsed_time(l1) / 10
+            lf_loss = (float(tr[0]), float(tr[-1]))
+            assert ctx.get_status() == 0
+            del scr_lf, labels0
         flops = 2.0 * ROWS * COLS * COLS
         extra["lfull_table"] = {"residual_ms_per_width": res_ms / nb, "gemm_ms_per_width": gemm_ms / nb,
                                 "table_ms_all_widths": res_ms + gemm_ms,
                                 "roofline": {"bound": "tensor", "kernel": "skim_lfull_gemm_kernel", "dtype": "fp16 in, fp32 accumulate",
                                              "achieved": flops / (gemm_ms / nb * 1e-3) / 1e12, "peak": tpeak, "peak_kind": f"of {tpeak_kind}",
                                              "unit": "TFLOP/s", "frac": flops / (gemm_ms / nb * 1e-3) / 1e12 / tpeak, "traffic": None},
-                                "note": "Section 3.4's L-full error for every row and width: 2*rows*cols^2 flop per width"}
+                                "scale_update_lfull_ms_per_adam_step": lf_step_ms, "scale_update_lfull_loss_first_last": lf_loss,
+                                "note": "Section 3.4's L-full error for every row and width: 2*rows*cols^2 flop per width; "
+                                        "the alpha-update on the same loss does one such contraction per Adam step"}
         del Hc, Dbuf, lf_scr
 
         # the optimum of the clustering objective per row (yardstick for the 50 Lloyd iterations)

@@ -21,6 +21,7 @@
  *   skim_scale_update     Adam steps on alpha with the labels fixed
  *                                                               (Algorithm 2, inner repeat)
  *   skim_cluster_rows_exact  the optimum of the clustering objective per row (yardstick for the iterations)
+ *   skim_scale_update_lfull  the same Adam steps on the L-full loss      (Section 4.3; Section 3.4)
  *   skim_residual, skim_err_lfull   the error of a row in the L-full form, (w - wq) X X^T (w - wq)^T
  *                                                               (Section 3.4; Section 4.2; Algorithm 3)
  *
@@ -321,6 +322,24 @@ int skim_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, 
 int skim_err_lfull_bytes(int64_t rows, int64_t cols, size_t *out);
 int skim_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
                    int64_t ldh, int exp2, void *scratch, size_t scratch_bytes, float *err, int64_t err_stride);
+
+/*
+ * skim_scale_update on the L-full loss (Section 4.3: "the loss calculation adopts the L-full form"; the form itself
+ * in Section 3.4):  loss = sum_i d_i H d_i^T,  d_ij = W_ij - alpha_j c_{i,l_ij},  with the importance-weighted centroids
+ * c of W * alpha^-1 re-fitted at every step as in skim_scale_update, and H = X X^T as for skim_err_lfull.  Per step the
+ * residual goes through the tensor-core contraction as binary16(float(d) * 2^exp2) (the gradient treats that
+ * rounding as the identity), Y = D H is kept in binary32, everything else is binary64.
+ *   labels, alpha, steps, lr0, decay, decay_every, loss_trace: as for skim_scale_update
+ *   H        [cols][ldh] binary16 (device), 16-byte aligned, ldh % 8 == 0
+ *   scratch  device, 256-byte aligned, at least skim_scale_lfull_bytes(rows, cols) bytes (6 bytes per element
+ *            for the residual and the product, plus the contraction's partial sums)
+ * cols % 8 == 0, ld % 8 == 0, W, importance and labels 16-byte aligned (SKIM_ERR_ALIGN otherwise).
+ */
+int skim_scale_lfull_bytes(int64_t rows, int64_t cols, size_t *out);
+int skim_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                            int64_t ld, const uint8_t *labels, const uint16_t *H, int64_t ldh, float *alpha, int steps,
+                            float lr0, float decay, int decay_every, int exp2, void *scratch, size_t scratch_bytes,
+                            double *loss_trace);
 
 /*
  * The whole path from HOST buffers: copies W and importance to the device staging area, runs

@@ -447,6 +447,37 @@ int skim_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols,
     return skim_launch_err_lfull(ctx, D, rows, cols, ldd, H, ldh, exp2, scratch, err, err_stride);
 }
 
+int skim_scale_lfull_bytes(int64_t rows, int64_t cols, size_t *out)
+{
+    if (!out) return SKIM_ERR_NULL;
+    if (rows < 1 || rows > 0x7fffff00 || cols < 8 || cols > 0x7fffff00) return SKIM_ERR_SHAPE;
+    *out = skim_scale_lfull_scratch_bytes(rows, cols);
+    return SKIM_OK;
+}
+
+int skim_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                            int64_t ld, const uint8_t *labels, const uint16_t *H, int64_t ldh, float *alpha, int steps,
+                            float lr0, float decay, int decay_every, int exp2, void *scratch, size_t scratch_bytes,
+                            double *loss_trace)
+{
+    if (!ctx || !W || !importance || !labels || !H || !alpha || !scratch) return SKIM_ERR_NULL;
+    int rc = check_matrix(ctx, rows, cols, ld);
+    if (rc) return rc;
+    if (rows < 1 || steps < 0 || decay_every < 1 || !(lr0 > 0.0f) || !(decay > 0.0f)) return SKIM_ERR_SHAPE;
+    if ((cols % 8) != 0 || (ld % 8) != 0 || ldh < cols || (ldh % 8) != 0 || exp2 < 0 || exp2 > 24) return SKIM_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(W) & 15u) || (reinterpret_cast<uintptr_t>(importance) & 15u) ||
+        (reinterpret_cast<uintptr_t>(labels) & 15u) || (reinterpret_cast<uintptr_t>(H) & 15u))
+        return SKIM_ERR_ALIGN;
+    rc = check_workspace(ctx, rows, cols);
+    if (rc) return rc;
+    if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0 || scratch_bytes < skim_scale_lfull_scratch_bytes(rows, cols))
+        return SKIM_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SKIM_ERR_CUDA;
+    return skim_launch_scale_update_lfull(ctx, W, importance, rows, cols, ld, labels, H, ldh, alpha, steps, lr0, decay,
+                                          decay_every, exp2, scratch, loss_trace);
+}
+
 // ---------------------------------------------------------------- host-buffer path
 
 namespace {

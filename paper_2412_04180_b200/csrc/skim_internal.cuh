@@ -153,8 +153,15 @@ int skim_launch_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t
                          const uint8_t *row_bits, int width, const SkimBits &bs, const float *s, int exp2, uint16_t *D,
                          int64_t ldd);
 size_t skim_lfull_scratch_bytes(int64_t rows, int64_t cols);
+// Y (optional): the product D H itself, [rows][ldy] binary32; err64 (optional): the row errors in binary64
 int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
-                          int64_t ldh, int exp2, void *scratch, float *err, int64_t err_stride);
+                          int64_t ldh, int exp2, void *scratch, float *err, int64_t err_stride, float *Y = nullptr,
+                          int64_t ldy = 0, double *err64 = nullptr);
+size_t skim_scale_lfull_scratch_bytes(int64_t rows, int64_t cols);
+int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                                   int64_t ld, const uint8_t *labels, const uint16_t *H, int64_t ldh, float *alpha,
+                                   int steps, float lr0, float decay, int decay_every, int exp2, void *scratch,
+                                   double *loss_trace);
 
 __host__ __device__ static inline int64_t skim_row_stride_words(int64_t cols, int b)
 {

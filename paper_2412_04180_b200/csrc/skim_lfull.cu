@@ -202,6 +202,8 @@ struct GemmArgs {
     int rows, cols;
     int mt, nt;              // tiles along rows and along columns
     float *partial;          // [mt * BM][nt]
+    float *Y;                // optional [rows][ldy]: the product D H itself (the scaling-vector update needs it)
+    int64_t ldy;
     unsigned long long *status;
 };
 
@@ -301,6 +303,13 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 }
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32), v);
+                if (a.Y && row < a.rows) {
+                    float *yrow = a.Y + (int64_t)row * a.ldy + col;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (col + u * 4 + 4 <= a.cols)
+                            *reinterpret_cast<uint4 *>(yrow + u * 4) = make_uint4(v[u * 4], v[u * 4 + 1], v[u * 4 + 2], v[u * 4 + 3]);
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const uint32_t w4[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
@@ -334,13 +343,14 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 }
 
 __global__ void skim_lfull_reduce_kernel(const float *__restrict__ partial, int rows, int nt, int exp2, float *__restrict__ err,
-                                         int64_t err_stride)
+                                         int64_t err_stride, double *__restrict__ err64)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows) return;
     double s = 0.0;
     for (int t = 0; t < nt; ++t) s += (double)partial[(int64_t)i * nt + t];
-    err[(int64_t)i * err_stride] = (float)ldexp(s, -2 * exp2);
+    if (err) err[(int64_t)i * err_stride] = (float)ldexp(s, -2 * exp2);
+    if (err64) err64[i] = ldexp(s, -2 * exp2);
 }
 
 int encode_map(CUtensorMap *map, const uint16_t *base, int64_t rows, int64_t cols, int64_t ld, int box_rows)
@@ -398,7 +408,8 @@ size_t skim_lfull_scratch_bytes(int64_t rows, int64_t cols)
 }
 
 int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
-                          int64_t ldh, int exp2, void *scratch, float *err, int64_t err_stride)
+                          int64_t ldh, int exp2, void *scratch, float *err, int64_t err_stride, float *Y, int64_t ldy,
+                          double *err64)
 {
     if (rows == 0) return SKIM_OK;
     CUtensorMap map_a, map_b;
@@ -414,13 +425,15 @@ int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_
     a.mt = (int)((rows + BM - 1) / BM);
     a.nt = (int)((cols + BN - 1) / BN);
     a.partial = (float *)scratch;
+    a.Y = Y;
+    a.ldy = ldy;
     a.status = (unsigned long long *)ctx->ws;
     SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lfull_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
     const int tiles = a.mt * a.nt;
     const unsigned blocks = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);    // persistent: one CTA per SM
     skim_lfull_gemm_kernel<<<blocks, GEMM_THREADS, GEMM_SMEM, ctx->stream>>>(map_a, map_b, a);
     SKIM_CUDA_OK(cudaGetLastError());
-    skim_lfull_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, ctx->stream>>>(a.partial, (int)rows, a.nt, exp2, err, err_stride);
+    skim_lfull_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, ctx->stream>>>(a.partial, (int)rows, a.nt, exp2, err, err_stride, err64);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 2;
     return SKIM_OK;

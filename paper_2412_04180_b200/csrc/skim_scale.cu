@@ -280,7 +280,254 @@ __global__ void skim_scale_finish_kernel(const double *__restrict__ alpha, int c
     if (j < cols) alpha32[j] = (float)alpha[j];
 }
 
+// ---------------------------------------------------------------- the same update on the L-full loss
+//
+//   loss(alpha) = sum_i d_i H d_i^T,  d_ij = W_ij - alpha_j c_{i,l_ij},  H = X X^T   (Section 4.3 with the L-full form of
+//   Section 3.4).  With Y = D H:  d loss / d alpha_j = sum_i -2 Y_ij c_{i,l} + q_{i,l} g_ij W_ij / alpha_j^2,
+//   q_ik = 2 R_ik / G_ik,  R_ik = sum_{j in k} Y_ij alpha_j.
+// Per Adam step: skim_scale_lf_residual_kernel (centroids of the step, residual as the binary16 operand of the
+// contraction), the tcgen05 GEMM of skim_lfull.cu (Y = D H stored, row-wise dot = the loss), skim_scale_lf_r_kernel
+// (R_ik, q_ik), skim_scale_lf_grad_kernel (column sums), and the Adam kernel above.
+
+struct ScaleLfArgs {
+    ScaleArgs s;
+    uint16_t *D;         // [rows][cols] binary16 residual * 2^exp2
+    const float *Y;      // [rows][cols] binary32, D H
+    int exp2;
+};
+
+// One warp per row: S_k = sum g w / alpha per cluster, c_k = S_k / G_k, then the row of D.
+__global__ void __launch_bounds__(SW * 32) skim_scale_lf_residual_kernel(ScaleLfArgs b)
+{
+    extern __shared__ __align__(16) double slots_all[];       // [SW][KC][32], then [SW][KC] centroids
+    const ScaleArgs &a = b.s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * SW + warp;
+    if (row >= a.rows) return;
+    double *slot = slots_all + (size_t)warp * (KC * 32) + lane;
+    double *cs = slots_all + (size_t)SW * (KC * 32) + warp * KC;
+#pragma unroll
+    for (int q = 0; q < KC; ++q) slot[q * 32] = 0.0;
+    Raw8 cur, nxt;
+    if (lane * 8 < a.cols) load8<true>(a, row, lane * 8, cur);
+    for (int e0 = lane * 8; e0 < a.cols; e0 += 256) {
+        if (e0 + 256 < a.cols) load8<true>(a, row, e0 + 256, nxt);
+        const uint32_t ww[4] = {cur.w.x, cur.w.y, cur.w.z, cur.w.w};
+        const float g[8] = {cur.ga.x, cur.ga.y, cur.ga.z, cur.ga.w, cur.gb.x, cur.gb.y, cur.gb.z, cur.gb.w};
+        const double al[8] = {cur.al[0].x, cur.al[0].y, cur.al[1].x, cur.al[1].y, cur.al[2].x, cur.al[2].y, cur.al[3].x, cur.al[3].y};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float wf = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+            const int l = (int)(((u < 4 ? cur.l.x : cur.l.y) >> (8 * (u & 3))) & (KC - 1));
+            slot[l * 32] += ((double)g[u] * (double)wf) * __drcp_rn(al[u]);
+        }
+        cur = nxt;
+    }
+    __syncwarp();
+    if (lane < KC) {
+        const double *base = slots_all + (size_t)warp * (KC * 32) + lane * 32;
+        double v = 0.0;
+        for (int t = 0; t < 32; ++t) v += base[(t + lane) & 31];
+        const double gk = a.tconst[row * KC + lane].x;
+        const double c = gk > 0.0 ? v / gk : 0.0;
+        cs[lane] = c;
+        a.tq[row * KC + lane] = make_double2(c, 0.0);
+    }
+    __syncwarp();
+    const float scale = __int_as_float((127 + b.exp2) << 23);
+    const uint16_t *Wr = a.W + row * a.ld;
+    const uint8_t *Lr = a.labels + row * (int64_t)a.cols;
+    uint16_t *Dr = b.D + row * (int64_t)a.cols;
+    for (int e0 = lane * 8; e0 < a.cols; e0 += 256) {
+        const uint4 wv = *reinterpret_cast<const uint4 *>(Wr + e0);
+        const uint2 lv = *reinterpret_cast<const uint2 *>(Lr + e0);
+        const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+        uint32_t out[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float wf = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+            const int l = (int)(((u < 4 ? lv.x : lv.y) >> (8 * (u & 3))) & (KC - 1));
+            const double d = (double)wf - a.alpha[e0 + u] * cs[l];
+            const uint32_t h = __half_as_ushort(__float2half_rn(__fmul_rn((float)d, scale)));
+            out[u >> 1] |= h << (16 * (u & 1));
+        }
+        *reinterpret_cast<uint4 *>(Dr + e0) = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+}
+
+// One warp per row: R_k = sum_{j in k} Y_ij alpha_j, q_k = 2 R_k / (2^exp2 G_k) into the row's table.
+__global__ void __launch_bounds__(SW * 32) skim_scale_lf_r_kernel(ScaleLfArgs b)
+{
+    extern __shared__ __align__(16) double slots_all[];       // [SW][KC][32]
+    const ScaleArgs &a = b.s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * SW + warp;
+    if (row >= a.rows) return;
+    double *slot = slots_all + (size_t)warp * (KC * 32) + lane;
+#pragma unroll
+    for (int q = 0; q < KC; ++q) slot[q * 32] = 0.0;
+    const float *Yr = b.Y + row * (int64_t)a.cols;
+    const uint8_t *Lr = a.labels + row * (int64_t)a.cols;
+    for (int e0 = lane * 8; e0 < a.cols; e0 += 256) {
+        const float4 ya = __ldcs(reinterpret_cast<const float4 *>(Yr + e0)), yb = __ldcs(reinterpret_cast<const float4 *>(Yr + e0 + 4));
+        const uint2 lv = __ldcs(reinterpret_cast<const uint2 *>(Lr + e0));
+        const float y[8] = {ya.x, ya.y, ya.z, ya.w, yb.x, yb.y, yb.z, yb.w};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int l = (int)(((u < 4 ? lv.x : lv.y) >> (8 * (u & 3))) & (KC - 1));
+            slot[l * 32] += (double)y[u] * a.alpha[e0 + u];
+        }
+    }
+    __syncwarp();
+    if (lane < KC) {
+        const double *base = slots_all + (size_t)warp * (KC * 32) + lane * 32;
+        double v = 0.0;
+        for (int t = 0; t < 32; ++t) v += base[(t + lane) & 31];
+        const double gk = a.tconst[row * KC + lane].x;
+        double2 cq = a.tq[row * KC + lane];
+        cq.y = gk > 0.0 ? ldexp(2.0 * v, -b.exp2) / gk : 0.0;
+        a.tq[row * KC + lane] = cq;
+    }
+}
+
+// A thread owns four columns and walks a range of rows: sum_i -2 Y_ij c + q g w / alpha_j^2.
+__global__ void __launch_bounds__(GT) skim_scale_lf_grad_kernel(ScaleLfArgs b)
+{
+    constexpr int RB = 8;
+    __shared__ double2 tq_s[RB * KC];
+    const ScaleArgs &a = b.s;
+    const int j0 = (blockIdx.x * GT + threadIdx.x) * GC;
+    const int64_t r0 = (int64_t)blockIdx.y * a.rows_per_range;
+    const int64_t r1 = min(a.rows, r0 + a.rows_per_range);
+    const double yscale = ldexp(1.0, -b.exp2);
+    double rr[GC], acc[GC];
+#pragma unroll
+    for (int u = 0; u < GC; ++u) {
+        const double al = j0 + u < a.cols ? a.alpha[j0 + u] : 1.0;
+        const double r = __drcp_rn(al);
+        rr[u] = r * r;
+        acc[u] = 0.0;
+    }
+    const bool in = j0 + GC <= a.cols;           // cols is a multiple of 8: a thread's columns are all inside or all outside
+    for (int64_t rb = r0; rb < r1; rb += RB) {
+        __syncthreads();
+        if (threadIdx.x < RB * KC && rb + threadIdx.x / KC < r1) tq_s[threadIdx.x] = a.tq[rb * KC + threadIdx.x];
+        uint2 wv[RB];
+        float4 gv[RB], yv[RB];
+        uint32_t lv[RB];
+#pragma unroll
+        for (int q = 0; q < RB; ++q) {
+            const int64_t row = rb + q;
+            wv[q] = make_uint2(0u, 0u); gv[q] = make_float4(0.f, 0.f, 0.f, 0.f); yv[q] = gv[q]; lv[q] = 0u;
+            if (row < r1 && in) {
+                wv[q] = __ldcs(reinterpret_cast<const uint2 *>(a.W + row * a.ld + j0));
+                gv[q] = __ldcs(reinterpret_cast<const float4 *>(a.G + row * a.ld + j0));
+                yv[q] = __ldcs(reinterpret_cast<const float4 *>(b.Y + row * (int64_t)a.cols + j0));
+                lv[q] = __ldcs(reinterpret_cast<const uint32_t *>(a.labels + row * (int64_t)a.cols + j0));
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < RB; ++q) {
+            if (rb + q >= r1) break;
+            const double2 *tq = tq_s + q * KC;
+            const uint32_t ww[2] = {wv[q].x, wv[q].y};
+            const float g[GC] = {gv[q].x, gv[q].y, gv[q].z, gv[q].w};
+            const float y[GC] = {yv[q].x, yv[q].y, yv[q].z, yv[q].w};
+#pragma unroll
+            for (int u = 0; u < GC; ++u) {
+                const double2 cq = tq[(lv[q] >> (8 * u)) & (KC - 1)];
+                const double wd = (double)__half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+                acc[u] += cq.y * (double)g[u] * wd * rr[u] - 2.0 * ((double)y[u] * yscale) * cq.x;
+            }
+        }
+    }
+    if (in) {
+#pragma unroll
+        for (int u = 0; u < GC; ++u) a.grad_part[(int64_t)blockIdx.y * a.cols + j0 + u] = acc[u];
+    }
+}
+
 }  // namespace
+
+size_t skim_scale_lfull_scratch_bytes(int64_t rows, int64_t cols)
+{
+    return skim_align256((size_t)rows * cols * 2) + skim_align256((size_t)rows * cols * 4) + skim_lfull_scratch_bytes(rows, cols);
+}
+
+int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
+                                   int64_t ld, const uint8_t *labels, const uint16_t *H, int64_t ldh, float *alpha,
+                                   int steps, float lr0, float decay, int decay_every, int exp2, void *scratch,
+                                   double *loss_trace)
+{
+    SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
+    const unsigned cb = (unsigned)((cols + 255) / 256);
+    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.adam_m, ws.adam_v, ws.status);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    ScaleLfArgs b;
+    ScaleArgs &a = b.s;
+    a.W = W;
+    a.G = importance;
+    a.labels = labels;
+    a.alpha = ws.alpha64;
+    a.rows = rows;
+    a.ld = ld;
+    a.cols = (int)cols;
+    a.vec = 1;
+    a.tconst = reinterpret_cast<double2 *>(ws.scale_const);
+    a.tq = reinterpret_cast<double2 *>(ws.scale_cq);
+    a.loss_row = ws.loss_part;
+    a.grad_part = ws.grad_part;
+    unsigned char *sp = (unsigned char *)scratch;
+    b.D = (uint16_t *)sp;
+    sp += skim_align256((size_t)rows * cols * 2);
+    float *Y = (float *)sp;
+    sp += skim_align256((size_t)rows * cols * 4);
+    void *gemm_scratch = sp;
+    b.Y = Y;
+    b.exp2 = exp2;
+    const int tiles = (int)((cols + GT * GC - 1) / (GT * GC));
+    int ranges = (4 * ctx->sm_count + tiles - 1) / tiles;
+    if (ranges > SKIM_SCALE_MAX_CTAS) ranges = SKIM_SCALE_MAX_CTAS;
+    if (ranges > rows) ranges = (int)rows;
+    a.rows_per_range = (int)((rows + ranges - 1) / ranges);
+    ranges = (int)((rows + a.rows_per_range - 1) / a.rows_per_range);
+    const size_t smem_init = (size_t)SW * NSUM * KC * 32 * sizeof(double);
+    const size_t smem_res = (size_t)SW * KC * 32 * sizeof(double) + (size_t)SW * KC * sizeof(double);
+    const size_t smem_r = (size_t)SW * KC * 32 * sizeof(double);
+    const unsigned sum_blocks = (unsigned)((rows + SW - 1) / SW);
+    SKIM_CUDA_OK(cudaFuncSetAttribute(skim_scale_sums_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_init));
+    skim_scale_sums_kernel<true, true><<<sum_blocks, SW * 32, smem_init, ctx->stream>>>(a);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    const double beta1 = 0.9, beta2 = 0.999, eps = 1e-8;
+    double p1 = 1.0, p2 = 1.0, lr = (double)lr0;
+    for (int t = 0; t < steps; ++t) {
+        if (t > 0 && t % decay_every == 0) lr *= (double)decay;
+        p1 *= beta1;
+        p2 *= beta2;
+        skim_scale_lf_residual_kernel<<<sum_blocks, SW * 32, smem_res, ctx->stream>>>(b);
+        SKIM_CUDA_OK(cudaGetLastError());
+        ctx->launches += 1;
+        const int rc = skim_launch_err_lfull(ctx, b.D, rows, cols, cols, H, ldh, exp2, gemm_scratch, nullptr, 1, Y, cols, ws.loss_part);
+        if (rc) return rc;
+        skim_scale_lf_r_kernel<<<sum_blocks, SW * 32, smem_r, ctx->stream>>>(b);
+        SKIM_CUDA_OK(cudaGetLastError());
+        skim_scale_lf_grad_kernel<<<dim3((unsigned)tiles, (unsigned)ranges), GT, 0, ctx->stream>>>(b);
+        SKIM_CUDA_OK(cudaGetLastError());
+        skim_scale_adam_kernel<<<cb + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
+                                                                ws.alpha64, ws.adam_m, ws.adam_v, lr, beta1, beta2,
+                                                                1.0 - p1, 1.0 - p2, eps,
+                                                                loss_trace ? loss_trace + t : nullptr);
+        SKIM_CUDA_OK(cudaGetLastError());
+        ctx->launches += 3;
+    }
+    skim_scale_finish_kernel<<<cb, 256, 0, ctx->stream>>>(ws.alpha64, (int)cols, alpha);
+    SKIM_CUDA_OK(cudaGetLastError());
+    ctx->launches += 1;
+    return SKIM_OK;
+}
 
 int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance, int64_t rows, int64_t cols,
                              int64_t ld, const uint8_t *labels, float *alpha, int steps, float lr0, float decay,

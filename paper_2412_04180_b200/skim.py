@@ -22,7 +22,7 @@ ERR_NAMES = {0: "SKIM_OK", -1: "SKIM_ERR_NULL", -2: "SKIM_ERR_SHAPE", -3: "SKIM_
 
 EXPORTS = ["skim_create", "skim_destroy", "skim_max_cols", "skim_workspace_bytes", "skim_set_workspace",
            "skim_apply_scale", "skim_cluster_rows", "skim_cluster_rows_at", "skim_cluster_exact_bytes", "skim_cluster_rows_exact", "skim_allocate_bits", "skim_allocate_bits_floor", "skim_allocate_bits_until", "skim_allocate_optimal_bytes", "skim_allocate_optimal",
-           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_residual", "skim_err_lfull_bytes", "skim_err_lfull", "skim_host_staging_bytes",
+           "skim_packed_layout", "skim_quantize", "skim_quantize_static", "skim_dequantize", "skim_matvec", "skim_scale_update", "skim_scale_lfull_bytes", "skim_scale_update_lfull", "skim_residual", "skim_err_lfull_bytes", "skim_err_lfull", "skim_host_staging_bytes",
            "skim_quantize_matrix_host", "skim_get_status", "skim_launch_count", "skim_kernel_timing",
            "skim_kernel_times", "skim_early_exit", "skim_lloyd_iterations", "skim_strerror"]
 
@@ -297,6 +297,27 @@ class Skim:
         _chk(lib().skim_scale_update(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
                                      C.c_int64(cols), _ptr(labels), _ptr(alpha), C.c_int(steps), C.c_float(lr0),
                                      C.c_float(decay), C.c_int(decay_every), _ptr(trace)), "skim_scale_update")
+        return trace[:steps] if want_trace else None
+
+    def scale_update_lfull(self, W, importance, labels, alpha, H, steps=120, lr0=0.01, decay=0.5, decay_every=40, exp2=8,
+                           want_trace=True, scratch=None):
+        """scale_update on the L-full loss with Gram matrix H (float16 [cols, cols]); alpha is updated in place."""
+        _dev(W, torch.float16, "W")
+        _dev(importance, torch.float32, "importance")
+        _dev(labels, torch.uint8, "labels")
+        _dev(alpha, torch.float32, "alpha")
+        _dev(H, torch.float16, "H")
+        rows, cols = W.shape
+        need = C.c_size_t()
+        _chk(lib().skim_scale_lfull_bytes(C.c_int64(rows), C.c_int64(cols), C.byref(need)), "skim_scale_lfull_bytes")
+        if scratch is None:
+            scratch = torch.empty(need.value, dtype=torch.uint8, device=W.device)
+        trace = torch.zeros(max(steps, 1), dtype=torch.float64, device=W.device) if want_trace else None
+        _chk(lib().skim_scale_update_lfull(self._h, _ptr(W), _ptr(importance), C.c_int64(rows), C.c_int64(cols),
+                                           C.c_int64(cols), _ptr(labels), _ptr(H), C.c_int64(H.stride(0)), _ptr(alpha),
+                                           C.c_int(steps), C.c_float(lr0), C.c_float(decay), C.c_int(decay_every),
+                                           C.c_int(exp2), _ptr(scratch), C.c_size_t(scratch.numel()), _ptr(trace)),
+             "skim_scale_update_lfull")
         return trace[:steps] if want_trace else None
 
     def residual(self, W, centroids, bit_set, width=None, row_bits=None, s=None, exp2=8, out=None):

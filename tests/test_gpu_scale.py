@@ -47,3 +47,46 @@ def test_scale_update_wide_rows(ctx, oracle):
                            alpha, steps=5)
     np.testing.assert_allclose(got.cpu().numpy(), trace, rtol=1e-7)
     np.testing.assert_allclose(alpha.cpu().numpy().astype(np.float64), want, rtol=1e-6)
+
+
+@pytest.mark.parametrize("rows,cols,steps", [(16, 64, 3), (40, 520, 12), (130, 264, 40), (300, 1000, 25)])
+def test_scale_update_lfull_matches_oracle(ctx, oracle, rows, cols, steps):
+    """The Adam steps on the L-full loss (Section 4.3).  Both sides round the residual to the same binary16 operand;
+    the GPU accumulates D H in binary32 on the tensor cores (relative error ~1e-6 of the magnitude sums) where the
+    oracle sums in binary64, so the loss is compared at 2e-5 (observed: 2e-6) and alpha, whose Adam steps turn a relative
+    gradient error delta into lr * delta per step, at 1e-4 relative + 1e-4 absolute (observed: 2e-5)."""
+    w, g = inputs.make_rows(rows, cols, 150 + rows, outlier_frac=0.01)
+    bits = (np.arange(rows) % 4 + 1).astype(np.uint8)
+    labels = _labels(oracle, w, g, bits)
+    H = inputs.make_gram(cols, 160 + cols)
+    a0 = inputs.make_scale(cols, 5, spread=0.05)
+    want, trace = oracle.scale_update_lfull(w, g, labels, a0.astype(np.float64), H, steps=steps)
+    ctx.reserve(rows, cols)
+    alpha = torch.from_numpy(a0.copy()).cuda()
+    got_trace = ctx.scale_update_lfull(torch.from_numpy(w).cuda(), torch.from_numpy(g).cuda(), torch.from_numpy(labels).cuda(),
+                                       alpha, torch.from_numpy(H).cuda(), steps=steps)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    got_trace = got_trace.cpu().numpy()
+    got = alpha.cpu().numpy().astype(np.float64)
+    print("max rel trace diff", np.max(np.abs(got_trace - trace) / trace), "max alpha diff", np.max(np.abs(got - want)))
+    np.testing.assert_allclose(got_trace, trace, rtol=2e-5)
+    np.testing.assert_allclose(got, want, rtol=1e-4, atol=1e-4)
+    assert trace[-1] < trace[0] or steps < 5
+
+
+def test_scale_update_lfull_argument_errors(ctx, skimlib):
+    rows, cols = 8, 64
+    w, g = inputs.make_rows(rows, cols, 3)
+    ctx.reserve(rows, cols)
+    W, G = torch.from_numpy(w).cuda(), torch.from_numpy(g).cuda()
+    L = torch.zeros((rows, cols), dtype=torch.uint8, device="cuda")
+    H = torch.eye(cols, dtype=torch.float16, device="cuda")
+    a = torch.ones(cols, device="cuda")
+    with pytest.raises(skimlib.SkimError) as e:
+        ctx.scale_update_lfull(W, G, L, a, H, steps=1, scratch=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -5
+    with pytest.raises(skimlib.SkimError) as e:
+        ctx.scale_update_lfull(W[:, :60].contiguous(), G[:, :60].contiguous(), L[:, :60].contiguous(), a[:60].contiguous(),
+                               H[:60, :60].contiguous(), steps=1)
+    assert e.value.code == -2
