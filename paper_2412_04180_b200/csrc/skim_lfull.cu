@@ -38,6 +38,7 @@ struct ResidualArgs {
     int cols;
     int nb, bmin, sumk;
     int exp2;
+    int vec;                 // rows of W, D (and of the scale vectors) allow 128-bit accesses
     uint16_t *D;
     unsigned long long *status;
 };
@@ -71,6 +72,39 @@ __global__ void __launch_bounds__(RES_T) skim_residual_kernel(ResidualArgs a)
     const uint16_t *Wr = a.W + row * a.ld;
     uint16_t *Dr = a.D + row * a.ldd;
     const float scale = __int_as_float((127 + a.exp2) << 23);       // 2^exp2, exact
+    if (a.vec) {
+        // eight elements per thread and step: one 128-bit load of W, one 128-bit store of D
+        for (int e0 = tid * 8; e0 < a.cols; e0 += RES_T * 8) {
+            const uint4 wv = __ldcs(reinterpret_cast<const uint4 *>(Wr + e0));
+            const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+            float rs[8], sv[8];
+            if (a.rscale) {
+                const float4 r0 = *reinterpret_cast<const float4 *>(a.rscale + e0), r1 = *reinterpret_cast<const float4 *>(a.rscale + e0 + 4);
+                rs[0] = r0.x; rs[1] = r0.y; rs[2] = r0.z; rs[3] = r0.w; rs[4] = r1.x; rs[5] = r1.y; rs[6] = r1.z; rs[7] = r1.w;
+            }
+            if (a.s) {
+                const float4 s0 = *reinterpret_cast<const float4 *>(a.s + e0), s1 = *reinterpret_cast<const float4 *>(a.s + e0 + 4);
+                sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w; sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
+            }
+            uint32_t out[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float w = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
+                float x = w;
+                if (a.rscale) x = __fmul_rn(w, rs[u]);
+                int code = (x > tf[7]) ? 8 : 0;
+                code += (x > tf[code + 3]) ? 4 : 0;
+                code += (x > tf[code + 1]) ? 2 : 0;
+                code += (x > tf[code]) ? 1 : 0;
+                float q = cs[code];
+                if (a.s) q = __fmul_rn(q, sv[u]);
+                const uint32_t h = __half_as_ushort(__float2half_rn(__fmul_rn(__fsub_rn(w, q), scale)));
+                out[u >> 1] |= h << (16 * (u & 1));
+            }
+            __stcs(reinterpret_cast<uint4 *>(Dr + e0), make_uint4(out[0], out[1], out[2], out[3]));
+        }
+        return;
+    }
     for (int e = tid; e < a.cols; e += RES_T) {
         const float w = __half2float(__ushort_as_half(Wr[e]));
         float x = w;
@@ -393,6 +427,8 @@ int skim_launch_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t
     a.bmin = bs.b_min;
     a.sumk = bs.sumk;
     a.exp2 = exp2;
+    a.vec = ((reinterpret_cast<uintptr_t>(W) & 15u) == 0 && (reinterpret_cast<uintptr_t>(D) & 15u) == 0 && ld % 8 == 0 &&
+             ldd % 8 == 0 && cols % 8 == 0 && (!s || (reinterpret_cast<uintptr_t>(s) & 15u) == 0)) ? 1 : 0;
     a.D = D;
     a.status = ws.status;
     skim_residual_kernel<<<(unsigned)rows, RES_T, 0, ctx->stream>>>(a);
