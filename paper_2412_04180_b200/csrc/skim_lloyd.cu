@@ -226,7 +226,9 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 Window win;
                 win.load(gi, ngi, gprev + 1 + gstep);     // centred where the boundary is heading
                 const int cnt = win.count_le(tf);
-                if ((cnt > 0 || win.ws == 0) && cnt < WIN) nle = win.ws + cnt;
+                // valid unless the boundary may lie outside the window: below its first entry (unless the window
+                // starts the index) or above its last (unless only padding follows)
+                if ((cnt > 0 || win.ws == 0) && (cnt < WIN || win.ws + WIN >= ngi)) nle = win.ws + cnt;
             }
             if (nle < 0) {
                 int lo = 0, hi = ngi;
