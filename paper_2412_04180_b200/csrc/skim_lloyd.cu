@@ -127,7 +127,11 @@ __device__ __forceinline__ void add_group(const G &grp, int n, double &s0, doubl
 // A window of 16 ascending group-index entries around the previous boundary position (at least 4
 // entries, i.e. 32 elements, on either side), read from shared memory with four independent loads;
 // only when the boundary left it does the search fall back to a binary search of the whole index.
-struct Window {
+template <bool HALF> struct Window;
+
+template <> struct Window<false> {
+    typedef float Entry;
+    static __device__ __forceinline__ bool le(float e, float t) { return e <= t; }
     float4 v[4];
     int ws;
     __device__ __forceinline__ void load(const float *gi, int ngi, int guess)   // gi: shared memory
@@ -154,6 +158,31 @@ struct Window {
     }
 };
 
+// The same window over a binary16 copy of the index (compact records: every value is a binary16 number, and a
+// binary16 value is <= t exactly when it is <= t rounded down to binary16): two loads, eight packed compares.
+template <> struct Window<true> {
+    typedef __half Entry;
+    static __device__ __forceinline__ bool le(__half e, float t) { return __half2float(e) <= t; }
+    uint4 v[2];
+    int ws;
+    __device__ __forceinline__ void load(const __half *gi, int ngi, int guess)   // gi: shared memory
+    {
+        ws = max(0, min((((guess + 4) >> 3) << 3) - 8, ngi - WIN));
+        const uint4 *p = reinterpret_cast<const uint4 *>(gi + ws);
+        v[0] = p[0];
+        v[1] = p[1];
+    }
+    __device__ __forceinline__ int count_le(float t) const
+    {
+        const __half2 th = __half2half2(__float2half_rd(t));
+        const uint32_t w[8] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w};
+        __half2 c = __hle2(*reinterpret_cast<const __half2 *>(&w[0]), th);
+#pragma unroll
+        for (int u = 1; u < 8; ++u) c = __hadd2(c, __hle2(*reinterpret_cast<const __half2 *>(&w[u]), th));
+        return (int)(__low2float(c) + __high2float(c));
+    }
+};
+
 // s1 / s0 for s0 > 0: binary32 reciprocal seed and two binary64 Newton corrections (relative
 // error about 2^-60, i.e. the correctly rounded quotient up to the last bit or so); operands far
 // outside the binary32 range take the plain division.
@@ -177,8 +206,8 @@ __device__ __forceinline__ double quotient(double s1, double s0)
 // prefix sums at the group start and the few elements in between.
 // On return sm.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
 template <bool HALF>
-__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float *gi, int nd, const ClusterArgs &a, int64_t row,
-                                           LloydSmem &sm)
+__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const typename Window<HALF>::Entry *gi, int nd,
+                                           const ClusterArgs &a, int64_t row, LloydSmem &sm)
 {
     const int lane = threadIdx.x & 31;
     const int m = a.m;
@@ -223,7 +252,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
         if (searches) {
             int nle = -1;                              // group-index entries <= tf
             if (gprev >= 0) {
-                Window win;
+                Window<HALF> win;
                 win.load(gi, ngi, gprev + 1 + gstep);     // centred where the boundary is heading
                 const int cnt = win.count_le(tf);
                 // valid unless the boundary may lie outside the window: below its first entry (unless the window
@@ -234,7 +263,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const float
                 int lo = 0, hi = ngi;
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
-                    if (gi[mid] <= tf) lo = mid + 1; else hi = mid;
+                    if (Window<HALF>::le(gi[mid], tf)) lo = mid + 1; else hi = mid;
                 }
                 nle = lo;
             }
@@ -335,7 +364,7 @@ template <bool HALF>
 __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(ClusterArgs a, int rows_in_chunk)
 {
     __shared__ LloydSmem sm_all[LLOYD_WARPS];
-    extern __shared__ __align__(16) float gi_all[];      // [LLOYD_WARPS][sk_entries(m)]
+    extern __shared__ __align__(16) unsigned char gi_all[];      // [LLOYD_WARPS][sk_entries(m)] index entries (binary32, or binary16 with compact records)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int local = blockIdx.x * LLOYD_WARPS + warp;
     if (local >= rows_in_chunk) return;
@@ -348,11 +377,20 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
     if (lane < 16) sm.dvals[lane] = reinterpret_cast<const float *>(rec + 64)[lane];
     // the row's group index, copied once
     const int nsk = sk_entries(a.m);
-    float *gi = gi_all + (size_t)warp * nsk;
+    typedef typename Window<HALF>::Entry Entry;
+    Entry *gi = reinterpret_cast<Entry *>(gi_all) + (size_t)warp * nsk;
     {
         const float4 *src = reinterpret_cast<const float4 *>(rec + row_record(a.m, HALF).gi);
-        float4 *dst = reinterpret_cast<float4 *>(gi);
-        for (int i = lane; i < nsk / 4; i += 32) dst[i] = __ldg(src + i);
+        for (int i = lane; i < nsk / 4; i += 32) {
+            const float4 v = __ldg(src + i);
+            if (HALF) {
+                // exact: the entries are binary16 numbers (the padding, the largest binary32, becomes +inf)
+                const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
+                reinterpret_cast<uint2 *>(gi)[i] = make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
+            } else {
+                reinterpret_cast<float4 *>(gi)[i] = v;
+            }
+        }
     }
     __syncwarp();
     lloyd_warp<HALF>(rec, gi, nd, a, row, sm);
@@ -366,7 +404,7 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
 int skim_launch_lloyd(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
 {
     const unsigned blocks = (unsigned)((rows + LLOYD_WARPS - 1) / LLOYD_WARPS);
-    const size_t smem = (size_t)LLOYD_WARPS * sk_entries(args.m) * sizeof(float);
+    const size_t smem = (size_t)LLOYD_WARPS * sk_entries(args.m) * (args.rec_half ? sizeof(__half) : sizeof(float));
     // set on every launch: a host-side call of microseconds, and no state shared between contexts
     void (*kernel)(ClusterArgs, int) = args.rec_half ? skim_lloyd_kernel<true> : skim_lloyd_kernel<false>;
     SKIM_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
