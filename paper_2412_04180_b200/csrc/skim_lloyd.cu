@@ -18,6 +18,15 @@ using namespace skimk;
 constexpr int LLOYD_WARPS = 4;   // rows per block
 constexpr int WIN = 16;          // group-index entries held in registers
 
+// dynamic shared memory of one warp: the group index (binary32, or binary16 with compact records), then 16 bytes
+// per segment and for the row totals
+__host__ __device__ inline size_t lloyd_warp_bytes(int m, bool half_index)
+{
+    const int nseg = ((((m + 7) >> 3) + (1 << SKIM_SEG_SHIFT) - 1) >> SKIM_SEG_SHIFT);
+    const size_t idx = ((size_t)sk_entries(m) * (half_index ? 2 : 4) + 15) & ~(size_t)15;
+    return idx + (size_t)(nseg + 1) * 16;
+}
+
 struct LloydSmem {
     double errs[32];
     float tfs[32];
@@ -206,8 +215,8 @@ __device__ __forceinline__ double quotient(double s1, double s0)
 // prefix sums at the group start and the few elements in between.
 // On return sm.tfs[L] holds the boundary (largest binary32 value still assigned to centroid L).
 template <bool HALF>
-__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const typename Window<HALF>::Entry *gi, int nd,
-                                           const ClusterArgs &a, int64_t row, LloydSmem &sm)
+__device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const typename Window<HALF>::Entry *gi, const double2 *segs,
+                                           int nd, const ClusterArgs &a, int64_t row, LloydSmem &sm)
 {
     const int lane = threadIdx.x & 31;
     const int m = a.m;
@@ -282,7 +291,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const typen
         double P0 = 0.0, P1 = 0.0, Pc = 0.0;
         if (normal) {
             if (searches) {
-                const double2 sb = __ldg(reinterpret_cast<const double2 *>(seg + (grp_i >> SKIM_SEG_SHIFT)));   // sums of the earlier segments
+                const double2 sb = segs[grp_i >> SKIM_SEG_SHIFT];   // sums of the earlier segments (shared memory)
                 P0 = sb.x + grp.p.x;
                 P1 = sb.y + grp.p.y;
                 if (final && !HALF) {
@@ -293,7 +302,7 @@ __device__ __forceinline__ void lloyd_warp(const unsigned char *rec, const typen
                 }
             } else {
                 // the last centroid of a width has no boundary above it: its prefix is the row total
-                const double2 tot = __ldg(reinterpret_cast<const double2 *>(seg + R.nseg));
+                const double2 tot = segs[R.nseg];
                 P0 = tot.x;
                 P1 = tot.y;
                 if (final && !HALF) Pc = __ldg(&seg[R.nseg].z);
@@ -378,8 +387,14 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
     // the row's group index, copied once
     const int nsk = sk_entries(a.m);
     typedef typename Window<HALF>::Entry Entry;
-    Entry *gi = reinterpret_cast<Entry *>(gi_all) + (size_t)warp * nsk;
+    const size_t per_warp = lloyd_warp_bytes(a.m, HALF);
+    Entry *gi = reinterpret_cast<Entry *>(gi_all + (size_t)warp * per_warp);
+    double2 *segs = reinterpret_cast<double2 *>(gi_all + (size_t)warp * per_warp + (((size_t)nsk * sizeof(Entry) + 15) & ~(size_t)15));
     {
+        // the segment table's sums of g and g*x (one pair per segment, the row totals last)
+        const RowRecord R = row_record(a.m, HALF);
+        const double4 *seg = reinterpret_cast<const double4 *>(rec + R.seg);
+        for (int i = lane; i <= R.nseg; i += 32) segs[i] = __ldg(reinterpret_cast<const double2 *>(seg + i));
         const float4 *src = reinterpret_cast<const float4 *>(rec + row_record(a.m, HALF).gi);
         for (int i = lane; i < nsk / 4; i += 32) {
             const float4 v = __ldg(src + i);
@@ -393,7 +408,7 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
         }
     }
     __syncwarp();
-    lloyd_warp<HALF>(rec, gi, nd, a, row, sm);
+    lloyd_warp<HALF>(rec, gi, segs, nd, a, row, sm);
     if (!a.codes) return;
     __syncwarp();
     write_codes(a, row, sm);
@@ -404,7 +419,7 @@ __global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(Cluster
 int skim_launch_lloyd(skim_ctx *ctx, const ClusterArgs &args, int64_t rows)
 {
     const unsigned blocks = (unsigned)((rows + LLOYD_WARPS - 1) / LLOYD_WARPS);
-    const size_t smem = (size_t)LLOYD_WARPS * sk_entries(args.m) * (args.rec_half ? sizeof(__half) : sizeof(float));
+    const size_t smem = (size_t)LLOYD_WARPS * lloyd_warp_bytes(args.m, args.rec_half != 0);
     // set on every launch: a host-side call of microseconds, and no state shared between contexts
     void (*kernel)(ClusterArgs, int) = args.rec_half ? skim_lloyd_kernel<true> : skim_lloyd_kernel<false>;
     SKIM_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
