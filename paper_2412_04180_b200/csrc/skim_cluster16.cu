@@ -196,9 +196,16 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
 
     // ---------------------------------------------------------------- pass 0: scan, claim slots, scatter
     {
+        // a thread's EPT consecutive counters go through 128-bit accesses (scalar ones would hit one bank 8 ways)
         uint32_t loc[EPT], s = 0, occupied = 0;
+        uint4 *C04 = reinterpret_cast<uint4 *>(C0 + tid * EPT);
 #pragma unroll
-        for (int u = 0; u < EPT; ++u) { loc[u] = C0[tid * EPT + u]; s += loc[u]; occupied += loc[u] ? 1u : 0u; }
+        for (int u = 0; u < EPT / 4; ++u) {
+            const uint4 v = C04[u];
+            loc[4 * u] = v.x; loc[4 * u + 1] = v.y; loc[4 * u + 2] = v.z; loc[4 * u + 3] = v.w;
+        }
+#pragma unroll
+        for (int u = 0; u < EPT; ++u) { s += loc[u]; occupied += loc[u] ? 1u : 0u; }
         // occupied low-digit bins: a lower bound of the number of distinct values
         occupied = __reduce_add_sync(0xffffffffu, occupied);
         if (lane == 0 && occupied) atomicAdd(&ps.misc[0], (int)occupied);
@@ -213,7 +220,14 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
         uint32_t run = inc - s;
         for (int w = 0; w < warp; ++w) run += scratch[w];
 #pragma unroll
-        for (int u = 0; u < EPT; ++u) { C0[tid * EPT + u] = run; run += loc[u]; }
+        for (int u = 0; u < EPT / 4; ++u) {
+            uint4 v;
+            v.x = run; run += loc[4 * u];
+            v.y = run; run += loc[4 * u + 1];
+            v.z = run; run += loc[4 * u + 2];
+            v.w = run; run += loc[4 * u + 3];
+            C04[u] = v;
+        }
     }
     __syncthreads();
 #pragma unroll
@@ -245,8 +259,18 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
     for (int d = warp; d < D1; d += NW) {
         uint32_t *cw = cnt1w + (d * THREADS) / 2 + lane * WPL;
         uint32_t wv[WPL], s = 0;
+        if constexpr (WPL % 4 == 0) {
 #pragma unroll
-        for (int u = 0; u < WPL; ++u) { wv[u] = cw[u]; s += (wv[u] & 0xffffu) + (wv[u] >> 16); }
+            for (int u = 0; u < WPL / 4; ++u) {
+                const uint4 v = reinterpret_cast<const uint4 *>(cw)[u];
+                wv[4 * u] = v.x; wv[4 * u + 1] = v.y; wv[4 * u + 2] = v.z; wv[4 * u + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < WPL; ++u) wv[u] = cw[u];
+        }
+#pragma unroll
+        for (int u = 0; u < WPL; ++u) s += (wv[u] & 0xffffu) + (wv[u] >> 16);
         uint32_t inc = s;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -258,8 +282,16 @@ __global__ void __launch_bounds__(THREADS, (THREADS <= 512 ? 2 : 1)) skim_sort16
 #pragma unroll
         for (int u = 0; u < WPL; ++u) {
             const uint32_t lo = wv[u] & 0xffffu, hi = wv[u] >> 16;
-            cw[u] = run | ((run + lo) << 16);
+            wv[u] = run | ((run + lo) << 16);
             run += lo + hi;
+        }
+        if constexpr (WPL % 4 == 0) {
+#pragma unroll
+            for (int u = 0; u < WPL / 4; ++u)
+                reinterpret_cast<uint4 *>(cw)[u] = make_uint4(wv[4 * u], wv[4 * u + 1], wv[4 * u + 2], wv[4 * u + 3]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < WPL; ++u) cw[u] = wv[u];
         }
     }
     // my stretch of positions, in order
