@@ -44,6 +44,7 @@ struct SkimWorkspace {
     float *rscale;               // [cols]     reciprocal of the installed scale vector
     int32_t *row_pos;            // [rows]     packed-row index of every source row
     double *alpha64;             // [cols]     scale-update master copy of alpha
+    double *alpha_il;            // [cols rounded up to 256]  the same values in the order the row-wise kernels load them
     double *adam_m;              // [cols]
     double *adam_v;              // [cols]
     double *loss_part;           // [rows]     scale update: loss of every row
@@ -77,6 +78,7 @@ static inline SkimWorkspace skim_carve(void *base, int64_t rows, int64_t cols)
     w.rscale = (float *)take((size_t)cols * 4);
     w.row_pos = (int32_t *)take((size_t)rows * 4);
     w.alpha64 = (double *)take((size_t)cols * 8);
+    w.alpha_il = (double *)take((((size_t)cols + 255) & ~(size_t)255) * 8);
     w.adam_m = (double *)take((size_t)cols * 8);
     w.adam_v = (double *)take((size_t)cols * 8);
     w.loss_part = (double *)take((size_t)(rows > SKIM_SCALE_MAX_CTAS ? rows : SKIM_SCALE_MAX_CTAS) * 8);

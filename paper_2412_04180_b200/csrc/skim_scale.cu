@@ -34,6 +34,7 @@ struct ScaleArgs {
     const float *G;
     const uint8_t *labels;
     const double *alpha;
+    const double *alpha_il; // alpha in the lane-interleaved order of alpha_il_pos()
     int64_t rows, ld;
     int cols;
     int vec;                // rows of W, G and labels allow the vector loads of both kernels
@@ -43,6 +44,16 @@ struct ScaleArgs {
     double *grad_part;      // [row ranges][cols]
     int rows_per_range;
 };
+
+// A lane of the row-wise kernels owns eight consecutive columns of every 256 and reads their alphas two at a
+// time.  From the plain array those reads are 64 bytes apart across the lanes (sixteen 128-byte wavefronts of the
+// L1 data path for 512 useful bytes, and that path is what bounds the sums kernel); from this order -- the u-th
+// pair of lane L at 64 u + 2 L of its block of 256 -- a warp's read is one contiguous 512 bytes.
+__host__ __device__ __forceinline__ int alpha_il_pos(int j)
+{
+    const int r = j & 255;
+    return (j & ~255) + 64 * ((r >> 1) & 3) + 2 * (r >> 3) + (r & 1);
+}
 
 // Eight consecutive elements of a row starting at e0 (a multiple of 8), as loaded; entries at or
 // beyond cols come back with zero importance, label 0 and alpha 1.
@@ -66,7 +77,7 @@ __device__ __forceinline__ void load8(const ScaleArgs &a, int64_t row, int e0, R
         r.gb = __ldcs(reinterpret_cast<const float4 *>(Gr + e0 + 4));
         r.l = __ldcs(reinterpret_cast<const uint2 *>(Lr + e0));
 #pragma unroll
-        for (int u = 0; u < 4; ++u) r.al[u] = __ldg(reinterpret_cast<const double2 *>(a.alpha + e0 + 2 * u));
+        for (int u = 0; u < 4; ++u) r.al[u] = __ldg(reinterpret_cast<const double2 *>(a.alpha_il + alpha_il_pos(e0 + 2 * u)));
     } else {
         uint32_t ww[4] = {0u, 0u, 0u, 0u}, ll[2] = {0u, 0u};
         float gg[8];
@@ -85,6 +96,34 @@ __device__ __forceinline__ void load8(const ScaleArgs &a, int64_t row, int e0, R
         r.l = make_uint2(ll[0], ll[1]);
 #pragma unroll
         for (int u = 0; u < 4; ++u) r.al[u] = make_double2(aa[2 * u], aa[2 * u + 1]);
+    }
+}
+
+// Adds four elements' terms to the lane's accumulator slots.  The four slots of a sum are read together
+// and the additions then run in element order in registers, an element whose cluster matches an earlier
+// one of the four continuing from that one's result: the same sums in the same order as one
+// read-modify-write after another, without the four round trips through shared memory in a row.
+template <int NS>
+__device__ __forceinline__ void add4(double *slot, const int (&l)[8], const double (&cs)[NS][8], int u0)
+{
+    double v[NS][4];
+#pragma unroll
+    for (int s = 0; s < NS; ++s)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[s][u] = slot[(s * KC + l[u0 + u]) * 32];
+    const bool e10 = l[u0 + 1] == l[u0], e20 = l[u0 + 2] == l[u0], e21 = l[u0 + 2] == l[u0 + 1];
+    const bool e30 = l[u0 + 3] == l[u0], e31 = l[u0 + 3] == l[u0 + 1], e32 = l[u0 + 3] == l[u0 + 2];
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        const double n0 = v[s][0] + cs[s][u0];
+        const double n1 = (e10 ? n0 : v[s][1]) + cs[s][u0 + 1];
+        const double n2 = (e21 ? n1 : e20 ? n0 : v[s][2]) + cs[s][u0 + 2];
+        const double n3 = (e32 ? n2 : e31 ? n1 : e30 ? n0 : v[s][3]) + cs[s][u0 + 3];
+        // in element order: where clusters repeat, the last store holds the full sum
+        slot[(s * KC + l[u0]) * 32] = n0;
+        slot[(s * KC + l[u0 + 1]) * 32] = n1;
+        slot[(s * KC + l[u0 + 2]) * 32] = n2;
+        slot[(s * KC + l[u0 + 3]) * 32] = n3;
     }
 }
 
@@ -107,22 +146,25 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
         const uint32_t ww[4] = {cur.w.x, cur.w.y, cur.w.z, cur.w.w};
         const float g[8] = {cur.ga.x, cur.ga.y, cur.ga.z, cur.ga.w, cur.gb.x, cur.gb.y, cur.gb.z, cur.gb.w};
         const double al[8] = {cur.al[0].x, cur.al[0].y, cur.al[1].x, cur.al[1].y, cur.al[2].x, cur.al[2].y, cur.al[3].x, cur.al[3].y};
+        int l[8];
+        double cs[INIT ? 2 : NSUM][8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const float wf = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
-            const int l = (int)(((u < 4 ? cur.l.x : cur.l.y) >> (8 * (u & 3))) & (KC - 1));
+            l[u] = (int)(((u < 4 ? cur.l.x : cur.l.y) >> (8 * (u & 3))) & (KC - 1));
             const double gd = (double)g[u], wd = (double)wf;
             const double gw = gd * wd;
-            double *sl = slot + l * 32;
             if (INIT) {
-                sl[0] += gd;
-                sl[KC * 32] += gw * wd;
+                cs[0][u] = gd;
+                cs[1][u] = gw * wd;
             } else {
-                sl[0] += gw * __drcp_rn(al[u]);
-                sl[KC * 32] += gw * al[u];
-                sl[2 * KC * 32] += gd * al[u] * al[u];
+                cs[0][u] = gw * __drcp_rn(al[u]);
+                cs[1][u] = gw * al[u];
+                cs[2][u] = gd * al[u] * al[u];
             }
         }
+        add4<INIT ? 2 : NSUM>(slot, l, cs, 0);
+        add4<INIT ? 2 : NSUM>(slot, l, cs, 4);
         cur = nxt;
     }
     __syncwarp();
@@ -233,8 +275,8 @@ __global__ void __launch_bounds__(GT) skim_scale_grad_kernel(ScaleArgs a)
 
 __global__ void __launch_bounds__(256) skim_scale_adam_kernel(const double *__restrict__ grad_part,
                                                                const double *__restrict__ loss_row, int nranges,
-                                                               int64_t rows, int cols, double *alpha, double *m1,
-                                                               double *m2, double lr, double beta1, double beta2,
+                                                               int64_t rows, int cols, double *alpha, double *alpha_il,
+                                                               double *m1, double *m2, double lr, double beta1, double beta2,
                                                                double bc1, double bc2, double eps, double *loss_out)
 {
     __shared__ double red[256];
@@ -259,10 +301,12 @@ __global__ void __launch_bounds__(256) skim_scale_adam_kernel(const double *__re
     const double a2 = beta2 * m2[j] + (1.0 - beta2) * g * g;
     m1[j] = a1;
     m2[j] = a2;
-    alpha[j] = alpha[j] - lr * (a1 / bc1) / (sqrt(a2 / bc2) + eps);
+    const double an = alpha[j] - lr * (a1 / bc1) / (sqrt(a2 / bc2) + eps);
+    alpha[j] = an;
+    alpha_il[alpha_il_pos(j)] = an;
 }
 
-__global__ void skim_scale_init_kernel(const float *__restrict__ alpha32, int cols, double *alpha,
+__global__ void skim_scale_init_kernel(const float *__restrict__ alpha32, int cols, double *alpha, double *alpha_il,
                                        double *m1, double *m2, unsigned long long *status)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -270,6 +314,7 @@ __global__ void skim_scale_init_kernel(const float *__restrict__ alpha32, int co
     const float v = alpha32[j];
     if (!(v > 0.0f) || v > 3.0e38f) atomicOr(status, (unsigned long long)SKIM_STATUS_BAD_SCALE);
     alpha[j] = (double)v;
+    alpha_il[alpha_il_pos(j)] = (double)v;
     m1[j] = 0.0;
     m2[j] = 0.0;
 }
@@ -462,7 +507,7 @@ int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float
 {
     SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
     const unsigned cb = (unsigned)((cols + 255) / 256);
-    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.adam_m, ws.adam_v, ws.status);
+    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, ws.status);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     ScaleLfArgs b;
@@ -471,6 +516,7 @@ int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float
     a.G = importance;
     a.labels = labels;
     a.alpha = ws.alpha64;
+    a.alpha_il = ws.alpha_il;
     a.rows = rows;
     a.ld = ld;
     a.cols = (int)cols;
@@ -517,7 +563,8 @@ int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float
         skim_scale_lf_grad_kernel<<<dim3((unsigned)tiles, (unsigned)ranges), GT, 0, ctx->stream>>>(b);
         SKIM_CUDA_OK(cudaGetLastError());
         skim_scale_adam_kernel<<<cb + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
-                                                                ws.alpha64, ws.adam_m, ws.adam_v, lr, beta1, beta2,
+                                                                ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, lr, beta1,
+                                                                beta2,
                                                                 1.0 - p1, 1.0 - p2, eps,
                                                                 loss_trace ? loss_trace + t : nullptr);
         SKIM_CUDA_OK(cudaGetLastError());
@@ -535,7 +582,7 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
 {
     SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
     const unsigned cb = (unsigned)((cols + 255) / 256);
-    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.adam_m, ws.adam_v, ws.status);
+    skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, ws.status);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
     ScaleArgs a;
@@ -543,6 +590,7 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
     a.G = importance;
     a.labels = labels;
     a.alpha = ws.alpha64;
+    a.alpha_il = ws.alpha_il;
     a.rows = rows;
     a.ld = ld;
     a.cols = (int)cols;
@@ -580,7 +628,8 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
         grad<<<dim3((unsigned)tiles, (unsigned)ranges), GT, 0, ctx->stream>>>(a);
         SKIM_CUDA_OK(cudaGetLastError());
         skim_scale_adam_kernel<<<cb + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
-                                                                ws.alpha64, ws.adam_m, ws.adam_v, lr, beta1, beta2,
+                                                                ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, lr, beta1,
+                                                                beta2,
                                                                 1.0 - p1, 1.0 - p2, eps,
                                                                 loss_trace ? loss_trace + t : nullptr);
         SKIM_CUDA_OK(cudaGetLastError());
