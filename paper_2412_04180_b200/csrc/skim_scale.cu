@@ -26,6 +26,7 @@ namespace {
 constexpr int KC = 16;      // clusters per row at most (4 bits)
 constexpr int SW = 4;       // warps (rows) per block of the sums kernel
 constexpr int NSUM = 3;
+constexpr int GW = 2;      // elements whose slot updates of the sums kernel go together
 constexpr int GT = 256;     // threads of a gradient block
 constexpr int GC = 4;       // columns per thread
 
@@ -99,31 +100,32 @@ __device__ __forceinline__ void load8(const ScaleArgs &a, int64_t row, int e0, R
     }
 }
 
-// Adds four elements' terms to the lane's accumulator slots.  The four slots of a sum are read together
-// and the additions then run in element order in registers, an element whose cluster matches an earlier
-// one of the four continuing from that one's result: the same sums in the same order as one
-// read-modify-write after another, without the four round trips through shared memory in a row.
-template <int NS>
-__device__ __forceinline__ void add4(double *slot, const int (&l)[8], const double (&cs)[NS][8], int u0)
+// Adds W (2 or 4) elements' terms to the lane's accumulator slots.  The slots of a sum are read together and the
+// additions then run in element order in registers, an element whose cluster matches an earlier one of the
+// group continuing from that one's result: the same sums in the same order as one read-modify-write after
+// another, without the round trips through shared memory in a row.
+template <int NS, int W>
+__device__ __forceinline__ void add_group(double *slot, const int (&l)[8], const double (&cs)[NS][8], int u0)
 {
-    double v[NS][4];
+    double v[NS][W];
 #pragma unroll
     for (int s = 0; s < NS; ++s)
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[s][u] = slot[(s * KC + l[u0 + u]) * 32];
-    const bool e10 = l[u0 + 1] == l[u0], e20 = l[u0 + 2] == l[u0], e21 = l[u0 + 2] == l[u0 + 1];
-    const bool e30 = l[u0 + 3] == l[u0], e31 = l[u0 + 3] == l[u0 + 1], e32 = l[u0 + 3] == l[u0 + 2];
+        for (int u = 0; u < W; ++u) v[s][u] = slot[(s * KC + l[u0 + u]) * 32];
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
-        const double n0 = v[s][0] + cs[s][u0];
-        const double n1 = (e10 ? n0 : v[s][1]) + cs[s][u0 + 1];
-        const double n2 = (e21 ? n1 : e20 ? n0 : v[s][2]) + cs[s][u0 + 2];
-        const double n3 = (e32 ? n2 : e31 ? n1 : e30 ? n0 : v[s][3]) + cs[s][u0 + 3];
+        double n[W];
+#pragma unroll
+        for (int u = 0; u < W; ++u) {
+            double base = v[s][u];
+#pragma unroll
+            for (int t = 0; t < u; ++t)
+                if (l[u0 + t] == l[u0 + u]) base = n[t];          // the latest earlier element of the cluster wins
+            n[u] = base + cs[s][u0 + u];
+        }
         // in element order: where clusters repeat, the last store holds the full sum
-        slot[(s * KC + l[u0]) * 32] = n0;
-        slot[(s * KC + l[u0 + 1]) * 32] = n1;
-        slot[(s * KC + l[u0 + 2]) * 32] = n2;
-        slot[(s * KC + l[u0 + 3]) * 32] = n3;
+#pragma unroll
+        for (int u = 0; u < W; ++u) slot[(s * KC + l[u0 + u]) * 32] = n[u];
     }
 }
 
@@ -163,8 +165,8 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
                 cs[2][u] = gd * al[u] * al[u];
             }
         }
-        add4<INIT ? 2 : NSUM>(slot, l, cs, 0);
-        add4<INIT ? 2 : NSUM>(slot, l, cs, 4);
+#pragma unroll
+        for (int u0 = 0; u0 < 8; u0 += GW) add_group<INIT ? 2 : NSUM, GW>(slot, l, cs, u0);
         cur = nxt;
     }
     __syncwarp();
@@ -200,11 +202,54 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_sums_kernel(ScaleArgs a)
     }
 }
 
+// The W, G and label entries of one thread's four columns in RB consecutive rows, as loaded.
+template <int RB>
+struct GradRows {
+    uint2 wv[RB];
+    float4 gv[RB];
+    uint32_t lv[RB];
+};
+
+template <bool VEC, int RB>
+__device__ __forceinline__ void grad_load(const ScaleArgs &a, int64_t rb, int64_t r1, int j0, bool full, GradRows<RB> &r)
+{
+#pragma unroll
+    for (int q = 0; q < RB; ++q) {
+        const int64_t row = rb + q;
+        r.wv[q] = make_uint2(0u, 0u); r.gv[q] = make_float4(0.f, 0.f, 0.f, 0.f); r.lv[q] = 0u;
+        if (row < r1 && j0 < a.cols) {
+            const uint16_t *Wr = a.W + row * a.ld + j0;
+            const float *Gr = a.G + row * a.ld + j0;
+            const uint8_t *Lr = a.labels + row * (int64_t)a.cols + j0;
+            if (full) {
+                r.wv[q] = __ldcs(reinterpret_cast<const uint2 *>(Wr));
+                r.gv[q] = __ldcs(reinterpret_cast<const float4 *>(Gr));
+                r.lv[q] = __ldcs(reinterpret_cast<const uint32_t *>(Lr));
+            } else {
+                uint32_t ww[2] = {0u, 0u};
+                float gg[GC];
+#pragma unroll
+                for (int u = 0; u < GC; ++u) {
+                    const bool in = j0 + u < a.cols;
+                    ww[u >> 1] |= (in ? (uint32_t)Wr[u] : 0u) << (16 * (u & 1));
+                    r.lv[q] |= (in ? (uint32_t)(Lr[u] & (KC - 1)) : 0u) << (8 * u);
+                    gg[u] = in ? Gr[u] : 0.0f;
+                }
+                r.wv[q] = make_uint2(ww[0], ww[1]);
+                r.gv[q] = make_float4(gg[0], gg[1], gg[2], gg[3]);
+            }
+        }
+    }
+}
+
 template <bool VEC>
 __global__ void __launch_bounds__(GT) skim_scale_grad_kernel(ScaleArgs a)
 {
-    constexpr int RB = 8;                       // rows whose loads are in flight together
-    __shared__ double2 tq_s[RB * KC];           // their (c_k, q_k) tables
+    // Rows go by in batches of RB.  While a batch is worked on, the next batch's loads are in flight and its
+    // (c_k, q_k) tables wait in a register of the first RB * KC threads; the tables alternate between two buffers,
+    // so one barrier per batch is enough.
+    constexpr int RB = 4;
+    __shared__ double2 tq_s[2][RB * KC];
     const int j0 = (blockIdx.x * GT + threadIdx.x) * GC;
     const int64_t r0 = (int64_t)blockIdx.y * a.rows_per_range;
     const int64_t r1 = min(a.rows, r0 + a.rows_per_range);
@@ -217,56 +262,37 @@ __global__ void __launch_bounds__(GT) skim_scale_grad_kernel(ScaleArgs a)
         acc[u] = 0.0;
     }
     const bool full = VEC && j0 + GC <= a.cols;
-    for (int64_t rb = r0; rb < r1; rb += RB) {
-        __syncthreads();                        // the previous batch's tables are no longer read
-        if (threadIdx.x < RB * KC && rb + threadIdx.x / KC < r1) tq_s[threadIdx.x] = a.tq[rb * KC + threadIdx.x];
-        uint2 wv[RB];
-        float4 gv[RB];
-        uint32_t lv[RB];
-#pragma unroll
-        for (int q = 0; q < RB; ++q) {
-            const int64_t row = rb + q;
-            wv[q] = make_uint2(0u, 0u); gv[q] = make_float4(0.f, 0.f, 0.f, 0.f); lv[q] = 0u;
-            if (row < r1 && j0 < a.cols) {
-                const uint16_t *Wr = a.W + row * a.ld + j0;
-                const float *Gr = a.G + row * a.ld + j0;
-                const uint8_t *Lr = a.labels + row * (int64_t)a.cols + j0;
-                if (full) {
-                    wv[q] = __ldcs(reinterpret_cast<const uint2 *>(Wr));
-                    gv[q] = __ldcs(reinterpret_cast<const float4 *>(Gr));
-                    lv[q] = __ldcs(reinterpret_cast<const uint32_t *>(Lr));
-                } else {
-                    uint32_t ww[2] = {0u, 0u};
-                    float gg[GC];
-#pragma unroll
-                    for (int u = 0; u < GC; ++u) {
-                        const bool in = j0 + u < a.cols;
-                        ww[u >> 1] |= (in ? (uint32_t)Wr[u] : 0u) << (16 * (u & 1));
-                        lv[q] |= (in ? (uint32_t)(Lr[u] & (KC - 1)) : 0u) << (8 * u);
-                        gg[u] = in ? Gr[u] : 0.0f;
-                    }
-                    wv[q] = make_uint2(ww[0], ww[1]);
-                    gv[q] = make_float4(gg[0], gg[1], gg[2], gg[3]);
-                }
-            }
+    const bool tq_thread = threadIdx.x < RB * KC;
+    GradRows<RB> cur, nxt;
+    grad_load<VEC, RB>(a, r0, r1, j0, full, cur);
+    if (tq_thread && r0 + threadIdx.x / KC < r1) tq_s[0][threadIdx.x] = a.tq[r0 * KC + threadIdx.x];
+    int buf = 0;
+    for (int64_t rb = r0; rb < r1; rb += RB, buf ^= 1) {
+        const int64_t rn = rb + RB;
+        double2 tnext = make_double2(0.0, 0.0);
+        if (rn < r1) {
+            grad_load<VEC, RB>(a, rn, r1, j0, full, nxt);
+            if (tq_thread && rn + threadIdx.x / KC < r1) tnext = a.tq[rn * KC + threadIdx.x];
         }
-        __syncthreads();
+        __syncthreads();                        // this batch's tables are in place; the other buffer is no longer read
 #pragma unroll
         for (int q = 0; q < RB; ++q) {
             const int64_t row = rb + q;
             if (row >= r1) break;
-            const double2 *tq = tq_s + q * KC;
-            const uint32_t ww[2] = {wv[q].x, wv[q].y};
-            const float g[GC] = {gv[q].x, gv[q].y, gv[q].z, gv[q].w};
+            const double2 *tq = tq_s[buf] + q * KC;
+            const uint32_t ww[2] = {cur.wv[q].x, cur.wv[q].y};
+            const float g[GC] = {cur.gv[q].x, cur.gv[q].y, cur.gv[q].z, cur.gv[q].w};
 #pragma unroll
             for (int u = 0; u < GC; ++u) {
-                const double2 cq = tq[(lv[q] >> (8 * u)) & (KC - 1)];
+                const double2 cq = tq[(cur.lv[q] >> (8 * u)) & (KC - 1)];
                 const double gd = (double)g[u];
                 const double wd = (double)__half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
                 const double res = wd - al[u] * cq.x;
                 acc[u] += gd * (cq.y * wd * rr[u] - 2.0 * cq.x * res);
             }
         }
+        if (tq_thread) tq_s[buf ^ 1][threadIdx.x] = tnext;
+        cur = nxt;
     }
 #pragma unroll
     for (int u = 0; u < GC; ++u)
@@ -293,10 +319,19 @@ __global__ void __launch_bounds__(256) skim_scale_adam_kernel(const double *__re
         if (threadIdx.x == 0 && loss_out) *loss_out = red[0];
         return;
     }
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= cols) return;
+    // 32 columns a block; the row ranges' partial gradients are dealt to 8 groups of threads, and the groups' sums
+    // are added in a fixed order
+    const int c = threadIdx.x & 31, sgrp = threadIdx.x >> 5;
+    const int j = blockIdx.x * 32 + c;
+    double gs = 0.0;
+    if (j < cols)
+        for (int b = sgrp; b < nranges; b += 8) gs += grad_part[(int64_t)b * cols + j];
+    red[threadIdx.x] = gs;
+    __syncthreads();
+    if (sgrp != 0 || j >= cols) return;
     double g = 0.0;
-    for (int b = 0; b < nranges; ++b) g += grad_part[(int64_t)b * cols + j];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) g += red[q * 32 + c];
     const double a1 = beta1 * m1[j] + (1.0 - beta1) * g;
     const double a2 = beta2 * m2[j] + (1.0 - beta2) * g * g;
     m1[j] = a1;
@@ -506,7 +541,7 @@ int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float
                                    double *loss_trace)
 {
     SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
-    const unsigned cb = (unsigned)((cols + 255) / 256);
+    const unsigned cb = (unsigned)((cols + 255) / 256), ab = (unsigned)((cols + 31) / 32);   // Adam: 32 columns a block
     skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, ws.status);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
@@ -562,7 +597,7 @@ int skim_launch_scale_update_lfull(skim_ctx *ctx, const uint16_t *W, const float
         SKIM_CUDA_OK(cudaGetLastError());
         skim_scale_lf_grad_kernel<<<dim3((unsigned)tiles, (unsigned)ranges), GT, 0, ctx->stream>>>(b);
         SKIM_CUDA_OK(cudaGetLastError());
-        skim_scale_adam_kernel<<<cb + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
+        skim_scale_adam_kernel<<<ab + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
                                                                 ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, lr, beta1,
                                                                 beta2,
                                                                 1.0 - p1, 1.0 - p2, eps,
@@ -581,7 +616,7 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
                              int decay_every, double *loss_trace)
 {
     SkimWorkspace ws = skim_carve(ctx->ws, rows, cols);
-    const unsigned cb = (unsigned)((cols + 255) / 256);
+    const unsigned cb = (unsigned)((cols + 255) / 256), ab = (unsigned)((cols + 31) / 32);   // Adam: 32 columns a block
     skim_scale_init_kernel<<<cb, 256, 0, ctx->stream>>>(alpha, (int)cols, ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, ws.status);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 1;
@@ -627,7 +662,7 @@ int skim_launch_scale_update(skim_ctx *ctx, const uint16_t *W, const float *impo
         SKIM_CUDA_OK(cudaGetLastError());
         grad<<<dim3((unsigned)tiles, (unsigned)ranges), GT, 0, ctx->stream>>>(a);
         SKIM_CUDA_OK(cudaGetLastError());
-        skim_scale_adam_kernel<<<cb + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
+        skim_scale_adam_kernel<<<ab + 1, 256, 0, ctx->stream>>>(ws.grad_part, ws.loss_part, ranges, rows, (int)cols,
                                                                 ws.alpha64, ws.alpha_il, ws.adam_m, ws.adam_v, lr, beta1,
                                                                 beta2,
                                                                 1.0 - p1, 1.0 - p2, eps,
