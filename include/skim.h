@@ -313,7 +313,8 @@ int skim_scale_update(skim_ctx *ctx, const uint16_t *W, const float *importance,
  *   scratch    device, 256-byte aligned, at least skim_err_lfull_bytes(rows, cols) bytes
  *   err        out binary32; err_stride elements between rows (n_bits to fill one column of the error table)
  * The products are exact in binary32 and are accumulated in binary32 by the tensor cores (cols terms per output
- * of D H, then cols terms per row), the per-tile sums in binary64:  |err - exact| <= (2 cols + 600) * 2^-24 *
+ * of D H, then cols terms per row), the sums per tile (per range of K where a tile of the last, partly filled round
+ * of tiles is cut along K) in binary64:  |err - exact| <= (2 cols + 600) * 2^-24 *
  * sum_jk |D_ij H_jk D_ik| / 4^exp2.  Needs the workspace (status word).
  */
 int skim_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t cols, int64_t ld, const float *centroids,

@@ -127,6 +127,7 @@ constexpr int STAGES = 4;
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int GEMM_THREADS = 192;
+constexpr int SPLIT_MAX = 8;                    // ranges of K a tile of the last round is cut into, at most
 constexpr int TMEM_COLS = 512;                  // two accumulator stages of BN binary32 columns
 constexpr long long WAIT_LIMIT_CYCLES = 400000000ll;   // about 0.2 s; a whole launch takes milliseconds
 constexpr size_t GEMM_SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
@@ -235,11 +236,34 @@ struct GemmArgs {
     int64_t ldd;
     int rows, cols;
     int mt, nt;              // tiles along rows and along columns
-    float *partial;          // [mt * BM][nt]
+    int full_tiles, split;   // tiles [full_tiles, mt * nt) are cut into `split` ranges of K (see unit_of)
+    float *partial;          // [mt * BM][split][nt]
     float *Y;                // optional [rows][ldy]: the product D H itself (the scaling-vector update needs it)
     int64_t ldy;
     unsigned long long *status;
 };
+
+// Work units.  Tiles are taken round-robin by the persistent CTAs; the tiles of the last, partly filled round
+// would leave most SMs idle for a whole tile time, so each of them is cut into `split` ranges of K that run
+// side by side.  The fused row-wise dot is linear in the accumulator, so a range simply leaves one more partial
+// dot per row (column `slice` of the partial array); the product Y itself is only written by unsplit launches.
+struct GemmUnit {
+    int tile, slice, kb0, kb1;
+};
+__device__ __forceinline__ GemmUnit unit_of(const GemmArgs &a, int u, int nkb)
+{
+    GemmUnit w;
+    if (u < a.full_tiles) {
+        w.tile = u; w.slice = 0; w.kb0 = 0; w.kb1 = nkb;
+    } else {
+        const int r = u - a.full_tiles;
+        w.tile = a.full_tiles + r / a.split;
+        w.slice = r % a.split;
+        w.kb0 = (int)((long long)nkb * w.slice / a.split);
+        w.kb1 = (int)((long long)nkb * (w.slice + 1) / a.split);
+    }
+    return w;
+}
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmArgs a)
@@ -251,6 +275,7 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (a.cols + BK - 1) / BK;
     const int ntiles = a.mt * a.nt;
+    const int nunits = a.full_tiles + (ntiles - a.full_tiles) * a.split;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&sy.full[s], 1); mbar_init(&sy.empty[s], 1); }
@@ -273,9 +298,10 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-                const int m0 = (t % a.mt) * BM, n0 = (t / a.mt) * BN;
-                for (int kb = 0; kb < nkb; ++kb) {
+            for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x) {
+                const GemmUnit w = unit_of(a, u, nkb);
+                const int m0 = (w.tile % a.mt) * BM, n0 = (w.tile / a.mt) * BN;
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     if (!(ok = mbar_wait(&sy.empty[stage], phase ^ 1u, abort_flag))) break;
                     unsigned char *sa = tiles + (size_t)stage * STAGE_BYTES;
                     mbar_expect_tx(&sy.full[stage], STAGE_BYTES);
@@ -292,18 +318,19 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             uint32_t phase = 0;
             bool ok = true;
             int it = 0;
-            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
+            for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x, ++it) {
+                const GemmUnit w = unit_of(a, u, nkb);
                 const int as = it & 1;
                 if (!(ok = mbar_wait(&sy.tmem_empty[as], (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(as * BN);
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
                     if (!(ok = mbar_wait(&sy.full[stage], phase, abort_flag))) break;
                     tc_fence_after();
                     const uint32_t sa = smem_u32(tiles + (size_t)stage * STAGE_BYTES), sb = sa + A_BYTES;
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_f16(tmem_d, umma_desc(sa + k * UMMA_K * 2), umma_desc(sb + k * UMMA_K * 2), (kb | k) ? 1u : 0u);
+                        umma_f16(tmem_d, umma_desc(sa + k * UMMA_K * 2), umma_desc(sb + k * UMMA_K * 2), (kb > w.kb0 || k) ? 1u : 0u);
                     umma_commit(&sy.empty[stage]);           // the stage is free once these MMAs have read it
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -315,9 +342,10 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const int q = warp & 3;                               // the tensor-memory lane quarter this warp may read
         bool ok = true;
         int it = 0;
-        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
+        for (int u = blockIdx.x; u < nunits && ok; u += gridDim.x, ++it) {
+            const GemmUnit w = unit_of(a, u, nkb);
             const int as = it & 1;
-            const int mb = t % a.mt, nb = t / a.mt;
+            const int mb = w.tile % a.mt, nb = w.tile / a.mt;
             const int row = mb * BM + q * 32 + lane;
             const int n0 = nb * BN;
             const uint16_t *drow = a.D + (int64_t)min(row, a.rows - 1) * a.ldd;
@@ -358,7 +386,7 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sy.tmem_empty[as]);
-            if (row < a.rows) a.partial[(int64_t)row * a.nt + nb] = acc;
+            if (row < a.rows) a.partial[((int64_t)row * a.split + w.slice) * a.nt + nb] = acc;
         }
     }
     // ---------------------------------------------------------------- teardown (every path comes here)
@@ -376,13 +404,19 @@ skim_lfull_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     }
 }
 
-__global__ void skim_lfull_reduce_kernel(const float *__restrict__ partial, int rows, int nt, int exp2, float *__restrict__ err,
-                                         int64_t err_stride, double *__restrict__ err64)
+// Adds a row's partial dots in a fixed order: slice 0 of every column tile, then the further slices of the tiles
+// that were cut along K (only those entries were written).
+__global__ void skim_lfull_reduce_kernel(const float *__restrict__ partial, int rows, int mt, int nt, int full_tiles, int split,
+                                         int exp2, float *__restrict__ err, int64_t err_stride, double *__restrict__ err64)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows) return;
+    const int mb = i / BM;
     double s = 0.0;
-    for (int t = 0; t < nt; ++t) s += (double)partial[(int64_t)i * nt + t];
+    for (int t = 0; t < nt; ++t) s += (double)partial[((int64_t)i * split) * nt + t];
+    for (int sl = 1; sl < split; ++sl)
+        for (int t = 0; t < nt; ++t)
+            if (t * mt + mb >= full_tiles) s += (double)partial[((int64_t)i * split + sl) * nt + t];
     if (err) err[(int64_t)i * err_stride] = (float)ldexp(s, -2 * exp2);
     if (err64) err64[i] = ldexp(s, -2 * exp2);
 }
@@ -440,7 +474,7 @@ int skim_launch_residual(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t
 size_t skim_lfull_scratch_bytes(int64_t rows, int64_t cols)
 {
     const int64_t mt = (rows + BM - 1) / BM, nt = (cols + BN - 1) / BN;
-    return skim_align256((size_t)(mt * BM) * (size_t)nt * sizeof(float));
+    return skim_align256((size_t)(mt * BM) * (size_t)nt * SPLIT_MAX * sizeof(float));
 }
 
 int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_t cols, int64_t ldd, const uint16_t *H,
@@ -466,10 +500,26 @@ int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_
     a.status = (unsigned long long *)ctx->ws;
     SKIM_CUDA_OK(cudaFuncSetAttribute(skim_lfull_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
     const int tiles = a.mt * a.nt;
-    const unsigned blocks = (unsigned)(tiles < ctx->sm_count ? tiles : ctx->sm_count);    // persistent: one CTA per SM
+    // the tiles of the last round, if it is not full, are cut along K into as many ranges as fit the SMs
+    const int nkb = (int)((cols + BK - 1) / BK);
+    const int rest = tiles % ctx->sm_count;
+    a.full_tiles = tiles;
+    a.split = 1;
+    if (!Y && rest > 0) {
+        int sp = ctx->sm_count / rest;
+        if (sp > SPLIT_MAX) sp = SPLIT_MAX;
+        if (sp > nkb) sp = nkb;
+        if (sp > 1) {
+            a.full_tiles = tiles - rest;
+            a.split = sp;
+        }
+    }
+    const int units = a.full_tiles + (tiles - a.full_tiles) * a.split;
+    const unsigned blocks = (unsigned)(units < ctx->sm_count ? units : ctx->sm_count);    // persistent: one CTA per SM
     skim_lfull_gemm_kernel<<<blocks, GEMM_THREADS, GEMM_SMEM, ctx->stream>>>(map_a, map_b, a);
     SKIM_CUDA_OK(cudaGetLastError());
-    skim_lfull_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, ctx->stream>>>(a.partial, (int)rows, a.nt, exp2, err, err_stride, err64);
+    skim_lfull_reduce_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, ctx->stream>>>(a.partial, (int)rows, a.mt, a.nt, a.full_tiles, a.split, exp2, err,
+                                                                                      err_stride, err64);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 2;
     return SKIM_OK;

@@ -97,6 +97,21 @@ def test_lfull_special_matrices(ctx, oracle):
     assert torch.equal(got2, got3)
 
 
+@pytest.mark.parametrize("cols", [968, 1160, 2560])
+def test_lfull_error_full_and_split_rounds(ctx, oracle, cols):
+    """4096 rows are 32 row tiles.  On a 148-SM part 968 columns give 128 tiles (one round, nothing cut), 1160
+    columns 160 tiles (one full round, the 12 tiles left cut into 8 ranges of K each), 2560 columns 320 tiles (two
+    full rounds, 24 tiles cut into 6 ranges): rows from full tiles and from cut tiles are compared with the oracle."""
+    rows = 4096
+    ctx.reserve(rows, cols)
+    rng = np.random.default_rng(cols)
+    D = (rng.standard_normal((rows, cols)) * 0.25).astype(np.float16)
+    H = inputs.make_gram(cols, 900 + cols)
+    sample = np.sort(rng.choice(rows, size=200, replace=False))
+    sample[0], sample[-1] = 0, rows - 1
+    _check_err(ctx, oracle, D, H, 0, rows=sample, label=f"cols={cols}")
+
+
 @pytest.mark.parametrize("cols,rows_total,seed", [(4096, 4096, 2000), (11008, 4096, 3001)])
 def test_lfull_table_at_llama_shapes(ctx, oracle, cols, rows_total, seed):
     """The L-full error table of a full-size matrix (the launch configuration the benchmark times), all four
