@@ -40,7 +40,7 @@ CLUSTER_BYTES_PER_ELEMENT = 6
 CLUSTER_BYTES_PER_ROW = 136
 # DRAM traffic of one launch of the dominant kernel per row, from the committed ncu capture
 # (bytes), or None when the kernel changed since the counters were taken.
-SORT_TRAFFIC_BYTES_PER_ROW = 136_611   # (135.38 MB read + 144.40 MB written) / 2048 rows, profiles/skim_sort16_kernel_2048x11008.md
+SORT_TRAFFIC_BYTES_PER_ROW = 136_638   # (135.38 MB read + 144.46 MB written) / 2048 rows, profiles/skim_sort16_kernel_2048x11008.md
 DOMINANT_KERNEL = "skim_sort16_kernel"
 DTYPE = "f64 sums, f32 centroid state (fp16 weights and fp32 importance in)"
 
