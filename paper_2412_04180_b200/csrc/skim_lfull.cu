@@ -506,9 +506,13 @@ int skim_launch_err_lfull(skim_ctx *ctx, const uint16_t *D, int64_t rows, int64_
     a.full_tiles = tiles;
     a.split = 1;
     if (!Y && rest > 0) {
-        int sp = ctx->sm_count / rest;
-        if (sp > SPLIT_MAX) sp = SPLIT_MAX;
-        if (sp > nkb) sp = nkb;
+        // `rest` tiles in s ranges each take ceil(rest s / SMs) sub-rounds of 1/s tile time: the least, the smaller s on a tie
+        int sp = 1;
+        double best = 1.0;
+        for (int c = 2; c <= SPLIT_MAX && c <= nkb; ++c) {
+            const double cost = (double)((rest * c + ctx->sm_count - 1) / ctx->sm_count) / c;
+            if (cost < best - 1e-9) { best = cost; sp = c; }
+        }
         if (sp > 1) {
             a.full_tiles = tiles - rest;
             a.split = sp;
