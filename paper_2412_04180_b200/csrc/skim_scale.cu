@@ -421,13 +421,20 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_lf_residual_kernel(ScaleLf
     for (int e0 = lane * 8; e0 < a.cols; e0 += 256) {
         const uint4 wv = *reinterpret_cast<const uint4 *>(Wr + e0);
         const uint2 lv = *reinterpret_cast<const uint2 *>(Lr + e0);
+        double al[8];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const double2 t = __ldg(reinterpret_cast<const double2 *>(a.alpha_il + alpha_il_pos(e0 + 2 * u)));
+            al[2 * u] = t.x;
+            al[2 * u + 1] = t.y;
+        }
         const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
         uint32_t out[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const float wf = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
             const int l = (int)(((u < 4 ? lv.x : lv.y) >> (8 * (u & 3))) & (KC - 1));
-            const double d = (double)wf - a.alpha[e0 + u] * cs[l];
+            const double d = (double)wf - al[u] * cs[l];
             const uint32_t h = __half_as_ushort(__float2half_rn(__fmul_rn((float)d, scale)));
             out[u >> 1] |= h << (16 * (u & 1));
         }
@@ -452,10 +459,17 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_lf_r_kernel(ScaleLfArgs b)
         const float4 ya = __ldcs(reinterpret_cast<const float4 *>(Yr + e0)), yb = __ldcs(reinterpret_cast<const float4 *>(Yr + e0 + 4));
         const uint2 lv = __ldcs(reinterpret_cast<const uint2 *>(Lr + e0));
         const float y[8] = {ya.x, ya.y, ya.z, ya.w, yb.x, yb.y, yb.z, yb.w};
+        double al[8];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const double2 t = __ldg(reinterpret_cast<const double2 *>(a.alpha_il + alpha_il_pos(e0 + 2 * u)));
+            al[2 * u] = t.x;
+            al[2 * u + 1] = t.y;
+        }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int l = (int)(((u < 4 ? lv.x : lv.y) >> (8 * (u & 3))) & (KC - 1));
-            slot[l * 32] += (double)y[u] * a.alpha[e0 + u];
+            slot[l * 32] += (double)y[u] * al[u];
         }
     }
     __syncwarp();
@@ -470,11 +484,36 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_lf_r_kernel(ScaleLfArgs b)
     }
 }
 
-// A thread owns four columns and walks a range of rows: sum_i -2 Y_ij c + q g w / alpha_j^2.
-__global__ void __launch_bounds__(GT) skim_scale_lf_grad_kernel(ScaleLfArgs b)
+// A thread owns four columns and walks a range of rows: sum_i -2 Y_ij c + q g w / alpha_j^2.  Batches of RB rows,
+// the next batch's loads in flight and its tables parked in registers, as in skim_scale_grad_kernel.
+template <int RB>
+struct GradRowsLf {
+    uint2 wv[RB];
+    float4 gv[RB], yv[RB];
+    uint32_t lv[RB];
+};
+
+template <int RB>
+__device__ __forceinline__ void grad_load_lf(const ScaleLfArgs &b, int64_t rb, int64_t r1, int j0, bool in, GradRowsLf<RB> &r)
 {
-    constexpr int RB = 8;
-    __shared__ double2 tq_s[RB * KC];
+    const ScaleArgs &a = b.s;
+#pragma unroll
+    for (int q = 0; q < RB; ++q) {
+        const int64_t row = rb + q;
+        r.wv[q] = make_uint2(0u, 0u); r.gv[q] = make_float4(0.f, 0.f, 0.f, 0.f); r.yv[q] = r.gv[q]; r.lv[q] = 0u;
+        if (row < r1 && in) {
+            r.wv[q] = __ldcs(reinterpret_cast<const uint2 *>(a.W + row * a.ld + j0));
+            r.gv[q] = __ldcs(reinterpret_cast<const float4 *>(a.G + row * a.ld + j0));
+            r.yv[q] = __ldcs(reinterpret_cast<const float4 *>(b.Y + row * (int64_t)a.cols + j0));
+            r.lv[q] = __ldcs(reinterpret_cast<const uint32_t *>(a.labels + row * (int64_t)a.cols + j0));
+        }
+    }
+}
+
+__global__ void __launch_bounds__(GT, 2) skim_scale_lf_grad_kernel(ScaleLfArgs b)
+{
+    constexpr int RB = 2;
+    __shared__ double2 tq_s[2][RB * KC];
     const ScaleArgs &a = b.s;
     const int j0 = (blockIdx.x * GT + threadIdx.x) * GC;
     const int64_t r0 = (int64_t)blockIdx.y * a.rows_per_range;
@@ -489,38 +528,35 @@ __global__ void __launch_bounds__(GT) skim_scale_lf_grad_kernel(ScaleLfArgs b)
         acc[u] = 0.0;
     }
     const bool in = j0 + GC <= a.cols;           // cols is a multiple of 8: a thread's columns are all inside or all outside
-    for (int64_t rb = r0; rb < r1; rb += RB) {
-        __syncthreads();
-        if (threadIdx.x < RB * KC && rb + threadIdx.x / KC < r1) tq_s[threadIdx.x] = a.tq[rb * KC + threadIdx.x];
-        uint2 wv[RB];
-        float4 gv[RB], yv[RB];
-        uint32_t lv[RB];
-#pragma unroll
-        for (int q = 0; q < RB; ++q) {
-            const int64_t row = rb + q;
-            wv[q] = make_uint2(0u, 0u); gv[q] = make_float4(0.f, 0.f, 0.f, 0.f); yv[q] = gv[q]; lv[q] = 0u;
-            if (row < r1 && in) {
-                wv[q] = __ldcs(reinterpret_cast<const uint2 *>(a.W + row * a.ld + j0));
-                gv[q] = __ldcs(reinterpret_cast<const float4 *>(a.G + row * a.ld + j0));
-                yv[q] = __ldcs(reinterpret_cast<const float4 *>(b.Y + row * (int64_t)a.cols + j0));
-                lv[q] = __ldcs(reinterpret_cast<const uint32_t *>(a.labels + row * (int64_t)a.cols + j0));
-            }
+    const bool tq_thread = threadIdx.x < RB * KC;
+    GradRowsLf<RB> cur, nxt;
+    grad_load_lf<RB>(b, r0, r1, j0, in, cur);
+    if (tq_thread && r0 + threadIdx.x / KC < r1) tq_s[0][threadIdx.x] = a.tq[r0 * KC + threadIdx.x];
+    int buf = 0;
+    for (int64_t rb = r0; rb < r1; rb += RB, buf ^= 1) {
+        const int64_t rn = rb + RB;
+        double2 tnext = make_double2(0.0, 0.0);
+        if (rn < r1) {
+            grad_load_lf<RB>(b, rn, r1, j0, in, nxt);
+            if (tq_thread && rn + threadIdx.x / KC < r1) tnext = a.tq[rn * KC + threadIdx.x];
         }
-        __syncthreads();
+        __syncthreads();                        // this batch's tables are in place; the other buffer is no longer read
 #pragma unroll
         for (int q = 0; q < RB; ++q) {
             if (rb + q >= r1) break;
-            const double2 *tq = tq_s + q * KC;
-            const uint32_t ww[2] = {wv[q].x, wv[q].y};
-            const float g[GC] = {gv[q].x, gv[q].y, gv[q].z, gv[q].w};
-            const float y[GC] = {yv[q].x, yv[q].y, yv[q].z, yv[q].w};
+            const double2 *tq = tq_s[buf] + q * KC;
+            const uint32_t ww[2] = {cur.wv[q].x, cur.wv[q].y};
+            const float g[GC] = {cur.gv[q].x, cur.gv[q].y, cur.gv[q].z, cur.gv[q].w};
+            const float y[GC] = {cur.yv[q].x, cur.yv[q].y, cur.yv[q].z, cur.yv[q].w};
 #pragma unroll
             for (int u = 0; u < GC; ++u) {
-                const double2 cq = tq[(lv[q] >> (8 * u)) & (KC - 1)];
+                const double2 cq = tq[(cur.lv[q] >> (8 * u)) & (KC - 1)];
                 const double wd = (double)__half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
                 acc[u] += cq.y * (double)g[u] * wd * rr[u] - 2.0 * ((double)y[u] * yscale) * cq.x;
             }
         }
+        if (tq_thread) tq_s[buf ^ 1][threadIdx.x] = tnext;
+        cur = nxt;
     }
     if (in) {
 #pragma unroll
