@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(SW * 32) skim_scale_lf_residual_kernel(ScaleLf
         for (int u = 0; u < 8; ++u) {
             const float wf = __half2float(__ushort_as_half((uint16_t)((u & 1) ? (ww[u >> 1] >> 16) : (ww[u >> 1] & 0xffffu))));
             const int l = (int)(((u < 4 ? cur.l.x : cur.l.y) >> (8 * (u & 3))) & (KC - 1));
-            slot[l * 32] += ((double)g[u] * (double)wf) * __drcp_rn(al[u]);
+            slot[l * 32] += ((double)g[u] * (double)wf) * rcp_pos(al[u]);
         }
         cur = nxt;
     }
