@@ -18,7 +18,8 @@
 //       cluster, read from the 512-byte table the first kernel left for the row), accumulated in
 //       registers; the row ranges leave partial gradients that the Adam kernel adds in a fixed order.
 //   skim_scale_adam_kernel  sums the partials and the rows' losses (deterministic), applies the
-//       Adam update to the binary64 master copy of alpha.
+//       Adam update to the binary64 master copy of alpha and to its lane-interleaved copy, the
+//       one the row-wise kernels read (alpha_il_pos).
 #include "skim_internal.cuh"
 
 namespace {
@@ -26,7 +27,7 @@ namespace {
 constexpr int KC = 16;      // clusters per row at most (4 bits)
 constexpr int SW = 4;       // warps (rows) per block of the sums kernel
 constexpr int NSUM = 3;
-constexpr int GW = 2;      // elements whose slot updates of the sums kernel go together
+constexpr int GW = 2;       // elements whose slot updates of the sums kernel go together
 constexpr int GT = 256;     // threads of a gradient block
 constexpr int GC = 4;       // columns per thread
 
