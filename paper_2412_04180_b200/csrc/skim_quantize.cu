@@ -4,10 +4,10 @@
 //
 //   skim_rank_rows_kernel  one block: stable partition of the rows by width -> packed position of
 //                          every row, row order, group starts and word offsets.
-//   skim_pack_kernel       one block per row: label = number of midpoints below the element,
-//                          8 labels per thread (packed fp16 compares, two weights per instruction,
-//                          when no scale is installed; a 4-step search in binary32 otherwise), four
-//                          threads merge their bit fields with shuffles and store whole words.
+//   skim_pack_kernel       one block per row: label = number of midpoints below the element
+//                          (packed fp16 compares, two weights per instruction, when no scale is
+//                          installed; a 4-step search in binary32 otherwise); a thread packs whole
+//                          groups of 32 elements into their b words.
 #include "skim_internal.cuh"
 
 namespace {
@@ -88,7 +88,6 @@ __global__ void __launch_bounds__(RT) skim_rank_rows_kernel(const uint8_t *__res
     }
 }
 
-constexpr int PT = 256;
 
 struct PackArgs {
     const uint16_t *W;
@@ -127,19 +126,109 @@ __device__ __forceinline__ uint32_t labels8_half(const uint4 raw, const __half2 
     return v;
 }
 
-__global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
+constexpr int PACK_MAX_THREADS = 384;   // three blocks of this size per SM at 56 registers
+
+// Labels of 8 elements starting at e0 on the general path (a scale vector installed, unaligned rows, or the ragged
+// end of a row): the clustered value in binary32, then a 4-step search of the binary32 thresholds.
+template <int B>
+__device__ __forceinline__ uint32_t labels8_general(const PackArgs &a, const uint16_t *Wr, int e0, const float *tf)
+{
+    float x[8];
+    if (a.vec_ok && e0 + 8 <= a.cols) {
+        const uint4 raw = *reinterpret_cast<const uint4 *>(Wr + e0);
+        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float2 f = __half22float2(h2[u]);
+            x[2 * u] = f.x;
+            x[2 * u + 1] = f.y;
+        }
+        if (a.rscale) {
+            const float4 r0 = *reinterpret_cast<const float4 *>(a.rscale + e0);
+            const float4 r1 = *reinterpret_cast<const float4 *>(a.rscale + e0 + 4);
+            x[0] = __fmul_rn(x[0], r0.x); x[1] = __fmul_rn(x[1], r0.y);
+            x[2] = __fmul_rn(x[2], r0.z); x[3] = __fmul_rn(x[3], r0.w);
+            x[4] = __fmul_rn(x[4], r1.x); x[5] = __fmul_rn(x[5], r1.y);
+            x[6] = __fmul_rn(x[6], r1.z); x[7] = __fmul_rn(x[7], r1.w);
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int e = e0 + u;
+            float xv = -__int_as_float(0x7f800000);    // past the row: label 0 (zero padding)
+            if (e < a.cols) {
+                xv = __half2float(__ushort_as_half(Wr[e]));
+                if (a.rscale) xv = __fmul_rn(xv, a.rscale[e]);
+            }
+            x[u] = xv;
+        }
+    }
+    uint32_t v = 0;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        int code = (x[u] > tf[7]) ? 8 : 0;
+        code += (x[u] > tf[code + 3]) ? 4 : 0;
+        code += (x[u] > tf[code + 1]) ? 2 : 0;
+        code += (x[u] > tf[code]) ? 1 : 0;
+        v |= (uint32_t)code << (u * B);
+    }
+    return v;
+}
+
+// One row at width B: a thread packs whole groups of 32 elements into their B words -- four 128-bit loads, the
+// labels of 8 elements at a time, the four 8B-bit fields joined with compile-time shifts -- so that no bits cross
+// threads (an earlier version gave a thread 8 elements and merged four threads' fields with 64-bit shuffles, which
+// cost more instructions than the compares).
+template <int B>
+__device__ __forceinline__ void pack_row(const PackArgs &a, const uint16_t *Wr, const __half2 *th, const float *tf,
+                                         uint32_t *dst, int64_t stride, bool fast)
+{
+    const int ngroups = (int)((stride + B - 1) / B);    // a group: 32 elements -> B words
+    for (int grp = threadIdx.x; grp < ngroups; grp += blockDim.x) {
+        const int e0 = grp * 32;
+        uint32_t v[4];
+        if (fast && e0 + 32 <= a.cols) {
+            uint4 raw[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) raw[q] = __ldg(reinterpret_cast<const uint4 *>(Wr + e0 + 8 * q));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = labels8_half<B>(raw[q], th);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = labels8_general<B>(a, Wr, e0 + 8 * q, tf);
+        }
+        uint32_t word[4] = {0u, 0u, 0u, 0u};
+        if constexpr (B == 4) {
+            word[0] = v[0]; word[1] = v[1]; word[2] = v[2]; word[3] = v[3];
+        } else if constexpr (B == 3) {
+            word[0] = v[0] | (v[1] << 24);
+            word[1] = (v[1] >> 8) | (v[2] << 16);
+            word[2] = (v[2] >> 16) | (v[3] << 8);
+        } else if constexpr (B == 2) {
+            word[0] = v[0] | (v[1] << 16);
+            word[1] = v[2] | (v[3] << 16);
+        } else {
+            word[0] = v[0] | (v[1] << 8) | (v[2] << 16) | (v[3] << 24);
+        }
+        const int64_t w0 = (int64_t)grp * B;
+        if (B == 4 && w0 + 4 <= stride) {
+            *reinterpret_cast<uint4 *>(dst + w0) = make_uint4(word[0], word[1], word[2], word[3]);   // rows start 16-byte aligned
+        } else {
+#pragma unroll
+            for (int w = 0; w < B; ++w)
+                if (w0 + w < stride) dst[w0 + w] = word[w];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(PACK_MAX_THREADS, 3) skim_pack_kernel(PackArgs a)
 {
     __shared__ float tf[16];
     __shared__ __half2 th_s[16];
     const int tid = threadIdx.x;
     const int64_t row = blockIdx.x;
     const uint16_t *Wr = a.W + row * a.ld;
-    const int quad = tid >> 2, ql = tid & 3;
-    // fp16 fast path: the weights of a step are loaded one step ahead; the first load goes out
-    // before the row's parameters are read
     const bool fast = a.vec_ok && !a.rscale;
-    uint4 ahead = make_uint4(0u, 0u, 0u, 0u);
-    if (fast && quad * 32 + ql * 8 + 8 <= a.cols) ahead = __ldg(reinterpret_cast<const uint4 *>(Wr + quad * 32 + ql * 8));
     const int pos = a.row_pos[row];
     if (pos < 0) return;
     const int b = (int)a.bits[row];
@@ -165,76 +254,26 @@ __global__ void __launch_bounds__(PT) skim_pack_kernel(PackArgs a)
     for (int j = 0; j < 15; ++j) th[j] = th_s[j];
     const int64_t stride = skim_row_stride_words(a.cols, b);
     uint32_t *dst = a.packed + a.group_info[a.nb + 1 + bi] + (int64_t)(pos - a.group_info[bi]) * stride;
-    const int ngroups = (int)((stride + b - 1) / b);   // a group: 32 elements -> b words
-    for (int base = 0; base < ngroups; base += PT / 4) {
-        const int grp = base + quad;
-        const int e0 = grp * 32 + ql * 8;
-        uint32_t v = 0;
-        const uint4 raw = ahead;
-        if (fast && base + PT / 4 < ngroups && e0 + (PT / 4) * 32 + 8 <= a.cols)
-            ahead = __ldg(reinterpret_cast<const uint4 *>(Wr + e0 + (PT / 4) * 32));
-        if (fast && e0 + 8 <= a.cols) {
-            switch (b) {
-            case 1: v = labels8_half<1>(raw, th); break;
-            case 2: v = labels8_half<2>(raw, th); break;
-            case 3: v = labels8_half<3>(raw, th); break;
-            default: v = labels8_half<4>(raw, th); break;
-            }
-        } else {
-            float x[8];
-            if (a.vec_ok && e0 + 8 <= a.cols) {
-                const uint4 raw = *reinterpret_cast<const uint4 *>(Wr + e0);
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float2 f = __half22float2(h2[u]);
-                    x[2 * u] = f.x;
-                    x[2 * u + 1] = f.y;
-                }
-                const float4 r0 = *reinterpret_cast<const float4 *>(a.rscale + e0);
-                const float4 r1 = *reinterpret_cast<const float4 *>(a.rscale + e0 + 4);
-                x[0] = __fmul_rn(x[0], r0.x); x[1] = __fmul_rn(x[1], r0.y);
-                x[2] = __fmul_rn(x[2], r0.z); x[3] = __fmul_rn(x[3], r0.w);
-                x[4] = __fmul_rn(x[4], r1.x); x[5] = __fmul_rn(x[5], r1.y);
-                x[6] = __fmul_rn(x[6], r1.z); x[7] = __fmul_rn(x[7], r1.w);
-            } else {
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int e = e0 + u;
-                    float xv = -__int_as_float(0x7f800000);    // past the row: label 0 (zero padding)
-                    if (e < a.cols) {
-                        xv = __half2float(__ushort_as_half(Wr[e]));
-                        if (a.rscale) xv = __fmul_rn(xv, a.rscale[e]);
-                    }
-                    x[u] = xv;
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                int code = (x[u] > tf[7]) ? 8 : 0;
-                code += (x[u] > tf[code + 3]) ? 4 : 0;
-                code += (x[u] > tf[code + 1]) ? 2 : 0;
-                code += (x[u] > tf[code]) ? 1 : 0;
-                v |= (uint32_t)code << (u * b);
-            }
-        }
-        const int sh = ql * 8 * b;                           // bit offset inside the group's b words
-        unsigned long long lo = 0ull, hi = 0ull;
-        if (sh < 64) {
-            lo = (unsigned long long)v << sh;
-            if (sh + 8 * b > 64) hi = (unsigned long long)v >> (64 - sh);
-        } else {
-            hi = (unsigned long long)v << (sh - 64);
-        }
-        lo |= __shfl_xor_sync(0xffffffffu, lo, 1);
-        hi |= __shfl_xor_sync(0xffffffffu, hi, 1);
-        lo |= __shfl_xor_sync(0xffffffffu, lo, 2);
-        hi |= __shfl_xor_sync(0xffffffffu, hi, 2);
-        const unsigned long long half = (ql < 2) ? lo : hi;
-        const uint32_t word = (uint32_t)(half >> (32 * (ql & 1)));
-        const int64_t widx = (int64_t)grp * b + ql;
-        if (grp < ngroups && ql < b && widx < stride) dst[widx] = word;
+    switch (b) {
+    case 1: pack_row<1>(a, Wr, th, tf, dst, stride, fast); break;
+    case 2: pack_row<2>(a, Wr, th, tf, dst, stride, fast); break;
+    case 3: pack_row<3>(a, Wr, th, tf, dst, stride, fast); break;
+    default: pack_row<4>(a, Wr, th, tf, dst, stride, fast); break;
     }
+}
+
+// Threads of a pack block: one per group of 32 elements of the longest packed row, in whole warps, at most
+// PACK_MAX_THREADS (longer rows take several groups per thread).
+static unsigned pack_threads(int64_t cols, const SkimBits &bs)
+{
+    int64_t most = 1;
+    for (int u = 0; u < bs.n_bits; ++u) {
+        const int b = bs.b_min + u;
+        const int64_t g = (skim_row_stride_words(cols, b) + b - 1) / b;
+        if (g > most) most = g;
+    }
+    const int64_t t = (most + 31) / 32 * 32;
+    return (unsigned)(t > PACK_MAX_THREADS ? PACK_MAX_THREADS : t);
 }
 
 __global__ void skim_reciprocal_kernel(const float *__restrict__ s, int64_t cols, float *__restrict__ r,
@@ -283,7 +322,7 @@ int skim_launch_quantize(skim_ctx *ctx, const uint16_t *W, int64_t rows, int64_t
     a.vec_ok = ((reinterpret_cast<uintptr_t>(W) & 15u) == 0 && (ld % 8) == 0) ? 1 : 0;
     a.packed = packed;
     a.lut = lut;
-    skim_pack_kernel<<<(unsigned)rows, PT, 0, ctx->stream>>>(a);
+    skim_pack_kernel<<<(unsigned)rows, pack_threads(cols, bs), 0, ctx->stream>>>(a);
     SKIM_CUDA_OK(cudaGetLastError());
     ctx->launches += 2;
     return SKIM_OK;
@@ -365,7 +404,7 @@ extern "C" int skim_quantize_static(void *cuda_stream, const uint16_t *W, int64_
     a.vec_ok = ((reinterpret_cast<uintptr_t>(W) & 15u) == 0 && (ld % 8) == 0) ? 1 : 0;
     a.packed = packed;
     a.lut = lut;
-    skim_pack_kernel<<<(unsigned)rows, PT, 0, stream>>>(a);
+    skim_pack_kernel<<<(unsigned)rows, pack_threads(cols, bs), 0, stream>>>(a);
     SKIM_CUDA_OK(cudaGetLastError());
     return SKIM_OK;
 }
