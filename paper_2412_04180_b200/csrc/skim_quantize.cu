@@ -230,8 +230,8 @@ __global__ void __launch_bounds__(PACK_MAX_THREADS, 3) skim_pack_kernel(PackArgs
     const uint16_t *Wr = a.W + row * a.ld;
     const bool fast = a.vec_ok && !a.rscale;
     const int pos = a.row_pos[row];
+    const int b = (int)a.bits[row];           // requested together with the position: one round trip, not two
     if (pos < 0) return;
-    const int b = (int)a.bits[row];
     const int bi = b - a.bmin;
     const int k = 1 << b;
     const int off = (1 << a.bmin) * ((1 << bi) - 1);
