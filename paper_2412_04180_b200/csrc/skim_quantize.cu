@@ -126,7 +126,10 @@ __device__ __forceinline__ uint32_t labels8_half(const uint4 raw, const __half2 
     return v;
 }
 
-constexpr int PACK_MAX_THREADS = 384;   // three blocks of this size per SM at 56 registers
+// Eight blocks of this size are resident per SM at 64 registers.  A block lives for little more than the two round
+// trips of its parameter loads, so many small resident blocks hide them better than few large ones (measured: 64,
+// 128, 192, 256 and 384 threads give 42.9, 40.0, 43.5, 44.3 and 45.8 us for rank + pack of 4096 x 11008).
+constexpr int PACK_MAX_THREADS = 128;
 
 // Labels of 8 elements starting at e0 on the general path (a scale vector installed, unaligned rows, or the ragged
 // end of a row): the clustered value in binary32, then a 4-step search of the binary32 thresholds.
@@ -181,16 +184,18 @@ __device__ __forceinline__ uint32_t labels8_general(const PackArgs &a, const uin
 // cost more instructions than the compares).
 template <int B>
 __device__ __forceinline__ void pack_row(const PackArgs &a, const uint16_t *Wr, const __half2 *th, const float *tf,
-                                         uint32_t *dst, int64_t stride, bool fast)
+                                         uint32_t *dst, int64_t stride, bool fast, uint4 (&raw)[4])
 {
     const int ngroups = (int)((stride + B - 1) / B);    // a group: 32 elements -> B words
+    // `raw` arrives holding the weights of the thread's first group (requested before the row's parameters were)
     for (int grp = threadIdx.x; grp < ngroups; grp += blockDim.x) {
         const int e0 = grp * 32;
         uint32_t v[4];
         if (fast && e0 + 32 <= a.cols) {
-            uint4 raw[4];
+            if (grp != (int)threadIdx.x) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) raw[q] = __ldg(reinterpret_cast<const uint4 *>(Wr + e0 + 8 * q));
+                for (int q = 0; q < 4; ++q) raw[q] = __ldg(reinterpret_cast<const uint4 *>(Wr + e0 + 8 * q));
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) v[q] = labels8_half<B>(raw[q], th);
         } else {
@@ -221,7 +226,7 @@ __device__ __forceinline__ void pack_row(const PackArgs &a, const uint16_t *Wr, 
     }
 }
 
-__global__ void __launch_bounds__(PACK_MAX_THREADS, 3) skim_pack_kernel(PackArgs a)
+__global__ void __launch_bounds__(PACK_MAX_THREADS, 8) skim_pack_kernel(PackArgs a)
 {
     __shared__ float tf[16];
     __shared__ __half2 th_s[16];
@@ -229,8 +234,17 @@ __global__ void __launch_bounds__(PACK_MAX_THREADS, 3) skim_pack_kernel(PackArgs
     const int64_t row = blockIdx.x;
     const uint16_t *Wr = a.W + row * a.ld;
     const bool fast = a.vec_ok && !a.rscale;
+    // the weights of the thread's first group and the row's two parameters are requested together; the codebook
+    // and the thresholds need the width, so they are one more round trip
+    uint4 raw[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) raw[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (fast && tid * 32 + 32 <= a.cols) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) raw[q] = __ldg(reinterpret_cast<const uint4 *>(Wr + tid * 32 + 8 * q));
+    }
     const int pos = a.row_pos[row];
-    const int b = (int)a.bits[row];           // requested together with the position: one round trip, not two
+    const int b = (int)a.bits[row];
     if (pos < 0) return;
     const int bi = b - a.bmin;
     const int k = 1 << b;
@@ -255,10 +269,10 @@ __global__ void __launch_bounds__(PACK_MAX_THREADS, 3) skim_pack_kernel(PackArgs
     const int64_t stride = skim_row_stride_words(a.cols, b);
     uint32_t *dst = a.packed + a.group_info[a.nb + 1 + bi] + (int64_t)(pos - a.group_info[bi]) * stride;
     switch (b) {
-    case 1: pack_row<1>(a, Wr, th, tf, dst, stride, fast); break;
-    case 2: pack_row<2>(a, Wr, th, tf, dst, stride, fast); break;
-    case 3: pack_row<3>(a, Wr, th, tf, dst, stride, fast); break;
-    default: pack_row<4>(a, Wr, th, tf, dst, stride, fast); break;
+    case 1: pack_row<1>(a, Wr, th, tf, dst, stride, fast, raw); break;
+    case 2: pack_row<2>(a, Wr, th, tf, dst, stride, fast, raw); break;
+    case 3: pack_row<3>(a, Wr, th, tf, dst, stride, fast, raw); break;
+    default: pack_row<4>(a, Wr, th, tf, dst, stride, fast, raw); break;
     }
 }
 
