@@ -50,31 +50,42 @@ __global__ void __launch_bounds__(RT) skim_rank_rows_kernel(const uint8_t *__res
         for (int v = 0; v < SKIM_MAX_NBITS; ++v) wsum[warp][v] = inc[v];
     }
     __syncthreads();
-    int before[SKIM_MAX_NBITS], total[SKIM_MAX_NBITS];
+    // warp 0 turns the warps' sums into exclusive prefixes; its last lane then holds the totals and lays out the groups
+    if (warp == 0) {
+        int x[SKIM_MAX_NBITS], run[SKIM_MAX_NBITS];
 #pragma unroll
-    for (int v = 0; v < SKIM_MAX_NBITS; ++v) {
-        before[v] = inc[v] - cnt[v];
-        total[v] = 0;
-        for (int w = 0; w < RT / 32; ++w) {
-            const int s = wsum[w][v];
-            if (w < warp) before[v] += s;
-            total[v] += s;
+        for (int v = 0; v < SKIM_MAX_NBITS; ++v) { x[v] = wsum[lane][v]; run[v] = x[v]; }
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+#pragma unroll
+            for (int v = 0; v < SKIM_MAX_NBITS; ++v) {
+                const int t = __shfl_up_sync(0xffffffffu, run[v], off);
+                if (lane >= off) run[v] += t;
+            }
         }
-    }
-    if (tid == 0) {
-        long long start = 0, word = 0;
-        for (int v = 0; v < nb; ++v) {
-            gstart[v] = (int)start;
-            group_info[v] = start;
-            group_info[nb + 1 + v] = word;
-            start += total[v];
-            word += (long long)total[v] * skim_row_stride_words(cols, bmin + v);
+#pragma unroll
+        for (int v = 0; v < SKIM_MAX_NBITS; ++v) wsum[lane][v] = run[v] - x[v];
+        if (lane == 31) {
+            long long start = 0, word = 0;
+#pragma unroll
+            for (int v = 0; v < SKIM_MAX_NBITS; ++v) {
+                if (v < nb) {
+                    gstart[v] = (int)start;
+                    group_info[v] = start;
+                    group_info[nb + 1 + v] = word;
+                    start += run[v];
+                    word += (long long)run[v] * skim_row_stride_words(cols, bmin + v);
+                }
+            }
+            gstart[nb] = (int)start;
+            group_info[nb] = start;
+            group_info[2 * nb + 1] = word;
         }
-        gstart[nb] = (int)start;
-        group_info[nb] = start;
-        group_info[2 * nb + 1] = word;
     }
     __syncthreads();
+    int before[SKIM_MAX_NBITS];
+#pragma unroll
+    for (int v = 0; v < SKIM_MAX_NBITS; ++v) before[v] = inc[v] - cnt[v] + wsum[warp][v];
     for (int64_t i = r0; i < r1; ++i) {
         const int u = (int)bits[i] - bmin;
         if (u < 0 || u >= nb) { row_pos[i] = -1; continue; }
