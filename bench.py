@@ -383,17 +383,20 @@ def run_ours(args):
             stream.synchronize()
             adam_ms = e0.elapsed_time(e1) / 40
             adam_bytes = 2 * 7 * ROWS * COLS          # two passes over fp16 W, fp32 importance and u8 labels
-            r0, r1, r2, r3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
-            r0.record(stream)
-            ctx.apply_scale(alpha)
-            _, labels, _ = ctx.cluster_rows_at(W, G, bits, BIT_SET, ITERS, want_codes=True, centroids=cent_at)
-            r1.record(stream)
-            ctx.scale_update(W, G, labels, alpha, steps=120, want_trace=False)
-            r2.record(stream)
-            ctx.apply_scale(alpha)
-            ctx.quantize(W, bits, cent_at, BIT_SET, out=out)
-            r3.record(stream)
-            stream.synchronize()
+            # two rounds, the second one reported: the first still meets one-time costs (allocator growth for the
+            # label matrix, lazily loaded kernels), which once showed as 14.6 ms instead of 2.1 ms of re-clustering
+            for _ in range(2):
+                r0, r1, r2, r3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+                r0.record(stream)
+                ctx.apply_scale(alpha)
+                _, labels, _ = ctx.cluster_rows_at(W, G, bits, BIT_SET, ITERS, want_codes=True, centroids=cent_at)
+                r1.record(stream)
+                ctx.scale_update(W, G, labels, alpha, steps=120, want_trace=False)
+                r2.record(stream)
+                ctx.apply_scale(alpha)
+                ctx.quantize(W, bits, cent_at, BIT_SET, out=out)
+                r3.record(stream)
+                stream.synchronize()
             ctx.apply_scale(None)
             assert ctx.get_status() == 0
         extra["scale_update"] = {"ms_per_adam_step": adam_ms, "algorithmic_bytes_per_step": adam_bytes,
@@ -402,7 +405,7 @@ def run_ours(args):
                                       "adam_120_steps_ms": r1.elapsed_time(r2), "emit_ms": r2.elapsed_time(r3),
                                       "total_ms": r0.elapsed_time(r3),
                                       "note": "one round of Algorithm 2 on the same matrix with the scale vector installed "
-                                              "(32-bit keys), labels written; single measurement, outside the timed region"}
+                                              "(32-bit keys), labels written; the second of two rounds, outside the timed region"}
         # the pipeline's own outputs again (the round above overwrote the packed form with the scaled one)
         step()
         stream.synchronize()
