@@ -359,8 +359,10 @@ __device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, c
         for (int bi = 0; bi < a.nb; ++bi) {
             const int k = 1 << (a.bmin + bi);
             if (only < 0 || only == bi) {
+                // number of boundaries below x: the boundaries of a width ascend, so log2(k) probes find it
                 int code = 0;
-                for (int u = 0; u < k - 1; ++u) code += (sm.tfs[off + u] < x) ? 1 : 0;
+                for (int step = k >> 1; step >= 1; step >>= 1)
+                    if (sm.tfs[off + code + step - 1] < x) code += step;
                 if (only < 0) a.codes[((int64_t)bi * a.rows + row) * m + e] = (uint8_t)code;
                 else a.codes[row * (int64_t)m + e] = (uint8_t)code;
             }
