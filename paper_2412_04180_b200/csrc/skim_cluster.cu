@@ -5,7 +5,7 @@
 // one warp per row, thousands of rows in flight) that iterates on the records.  The split exists
 // because the Lloyd iteration is a long chain of dependent small steps: inside the sort block it ran
 // on one warp while two rows filled an SM's shared memory; from global memory (the hot lines stay in
-// L1) every SM keeps 32 rows in flight.
+// L1) every SM keeps 28 rows in flight.
 //
 // This file: the generic sort kernel, which handles every case -- scaled rows (32-bit keys of the
 // binary32 product) and rows whose layout rules out the vectorised fp16-key kernel of

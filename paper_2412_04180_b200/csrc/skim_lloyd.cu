@@ -371,8 +371,10 @@ __device__ __forceinline__ void write_codes(const ClusterArgs &a, int64_t row, c
     }
 }
 
+// Seven blocks of four rows per SM: an eighth would hold the kernel to 64 registers, which measured slower on every
+// shape (the full-record form spills there).
 template <bool HALF>
-__global__ void __launch_bounds__(LLOYD_WARPS * 32, 8) skim_lloyd_kernel(ClusterArgs a, int rows_in_chunk)
+__global__ void __launch_bounds__(LLOYD_WARPS * 32, 7) skim_lloyd_kernel(ClusterArgs a, int rows_in_chunk)
 {
     __shared__ LloydSmem sm_all[LLOYD_WARPS];
     extern __shared__ __align__(16) unsigned char gi_all[];      // [LLOYD_WARPS][sk_entries(m)] index entries (binary32, or binary16 with compact records)
