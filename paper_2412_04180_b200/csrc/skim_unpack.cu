@@ -103,16 +103,21 @@ __device__ __forceinline__ void unpack_row(const UnpackArgs &a, const float *vec
             if (t >= steps) break;
             const uint32_t codes = lane_codes<B>(wv[q], lane);
             const int j0 = t * STEP + lane * 8;
-            // the step's 256 vector entries are stored as two runs of quads (see vec_slot): both loads are conflict-free
-            const float4 va = *reinterpret_cast<const float4 *>(vec + t * STEP + lane * 4);
-            const float4 vb = *reinterpret_cast<const float4 *>(vec + t * STEP + 128 + lane * 4);
+            // the step's 256 vector entries are stored as two runs of quads (see vec_slot): both loads are conflict-free;
+            // a dequantiser without a scaling vector has nothing to multiply by and skips them
+            const bool use_vec = MATVEC || a.s != nullptr;
+            float4 va = make_float4(1.f, 1.f, 1.f, 1.f), vb = va;
+            if (use_vec) {
+                va = *reinterpret_cast<const float4 *>(vec + t * STEP + lane * 4);
+                vb = *reinterpret_cast<const float4 *>(vec + t * STEP + 128 + lane * 4);
+            }
             const float v[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
             float r[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const float e = book[(codes >> (u * B)) & ((1u << B) - 1u)];
                 if (MATVEC) acc = fmaf(e, v[u], acc);
-                else r[u] = __fmul_rn(e, v[u]);
+                else r[u] = use_vec ? __fmul_rn(e, v[u]) : e;
             }
             if (!MATVEC) {
                 uint16_t *dst = a.out + src_row * a.ld + j0;
@@ -145,7 +150,7 @@ __global__ void __launch_bounds__(UT) skim_unpack_kernel(UnpackArgs a)
 {
     extern __shared__ __align__(16) float vec[];          // [cols rounded up to STEP], zero beyond cols
     __shared__ float books[UW][16];
-    const int padded = (a.cols + STEP - 1) / STEP * STEP;
+    const int padded = (MATVEC || a.s) ? (a.cols + STEP - 1) / STEP * STEP : 0;
     for (int j = threadIdx.x; j < padded; j += UT) {
         float v = 0.0f;
         if (j < a.cols) {
